@@ -1,0 +1,179 @@
+/*
+ * think.h -- C ABI of the ThinK hot path (query-driven key-cache channel pruning)
+ * for NVIDIA B200 (sm_100a).
+ *
+ * Problem statement (paper, Sec. 1 and Sec. 3.1): the key and value caches are
+ * tensors K, V in R^{B x S x L x N x D} (batch, tokens, layers, heads, head
+ * dimension).  Given a pruning ratio lambda, T = floor((1 - lambda) D) key
+ * channels are kept per head (Sec. 3.1, Eq. 2); the channels are chosen by the
+ * query-driven score of Sec. 3.2 evaluated with the last S_obs queries
+ * ("Observation Window"); the most recent S_recent prompt tokens and all newly
+ * decoded tokens keep all D key channels (Sec. 3.3).
+ *
+ * Call order:   thinK_cache_bytes -> thinK_create -> thinK_score_select ->
+ *               thinK_compact -> { thinK_append -> thinK_decode_attn }* -> thinK_destroy
+ *
+ * Conventions that hold for every entry point
+ *  - All tensor pointers are DEVICE pointers unless marked "host".  The caller
+ *    allocates and owns every device buffer; the library never allocates device
+ *    memory and never frees anything but its own host-side handle.
+ *  - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and
+ *    return without synchronising.  Calls on one handle must be stream-ordered
+ *    with respect to each other.
+ *  - Errors are return codes.  Arguments are validated on the host before any
+ *    launch; an invalid call launches nothing.  Inputs are assumed finite
+ *    (NaN/Inf in K or Q leaves the selection unspecified).
+ *  - Element type (`dtype`): bf16 or fp32 for K, V, Q, q, k_new, v_new and out.
+ */
+#ifndef THINK_H_
+#define THINK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  THINK_OK = 0,
+  THINK_ERR_INVALID_ARG = 1, /* null / misaligned pointer, bad shape, bad layer range */
+  THINK_ERR_UNSUPPORTED = 2, /* head dimension, group size or dtype without a kernel */
+  THINK_ERR_STATE = 3,       /* call out of order */
+  THINK_ERR_CAPACITY = 4,    /* tail full (max_new_tokens) or buffer too small */
+  THINK_ERR_CUDA = 5         /* a CUDA runtime call or launch failed */
+} thinK_status;
+
+typedef enum { THINK_BF16 = 0, THINK_F32 = 1 } thinK_dtype;
+
+/* Score used to rank the channels of a key head. */
+typedef enum {
+  THINK_SCORE_QUERY_DRIVEN = 0, /* Sec. 3.2: ||Q[-S_obs:, j] K[:, j]^T||_F                      */
+  THINK_SCORE_KEY_L2 = 1,       /* Sec. 3.1, Eq. 1 with p = 2: ||K[:, j]||_2 (paper's baseline) */
+  THINK_SCORE_KEY_L1 = 2        /* Sec. 3.1, Eq. 1 with p = 1: ||K[:, j]||_1                    */
+} thinK_criterion;
+
+typedef struct {
+  int32_t B;              /* batch entries */
+  int32_t L;              /* layers held by this cache */
+  int32_t N_q;            /* query heads; N_q % N_kv == 0, group size G = N_q / N_kv in {1,2,4,8} */
+  int32_t N_kv;           /* key/value heads */
+  int32_t D;              /* head dimension: 64 or 128 */
+  int32_t S_max;          /* rows allocated along S in K and V (>= every seq_len) */
+  int32_t S_obs;          /* observation window (Sec. 3.2); seq_len >= S_obs */
+  int32_t S_recent;       /* prompt tokens left unpruned (Sec. 3.3, Sec. 4.3 "recent size") */
+  int32_t max_new_tokens; /* decode steps the unpruned tail can take */
+  int32_t dtype;          /* thinK_dtype */
+  int32_t criterion;      /* thinK_criterion */
+  int32_t reserved;       /* 0 */
+  double lambda;          /* pruning ratio, 0 <= lambda < 1 */
+} thinK_config;
+
+/* A strided view of a B x S x L x N x D tensor.  Strides are in ELEMENTS; the D
+ * axis is contiguous.  `ptr` and every stride must be multiples of 16 bytes.
+ * The paper's layout is stride_b = S*L*N*D, stride_s = L*N*D, stride_l = N*D,
+ * stride_n = D; a per-layer cache [B, N, S, D] is expressed by other strides. */
+typedef struct {
+  void* ptr;
+  int64_t stride_b, stride_s, stride_l, stride_n;
+} thinK_tensor5;
+
+/* Byte sizes of the caller-allocated device buffers (each 256-byte aligned). */
+typedef struct {
+  size_t k_thin;    /* pruned prefix keys, library layout (below) */
+  size_t tail_k;    /* unpruned keys: recent prompt rows + decoded tokens */
+  size_t tail_v;    /* values of the same tokens, [B, L, N_kv, cap, D] */
+  size_t idx;       /* kept channels, uint8 [B, L, N_kv, T], ascending */
+  size_t scores;    /* channel scores, fp64 [B, L, N_kv, D] */
+  size_t workspace; /* reduction partials, split-softmax states, counters */
+  /* The paper's accounting of the same cache (Sec. 3.1, Sec. 3.3), in bytes:
+   * keys of the pruned prefix at T channels + unpruned keys at D + all values,
+   * with the tail at full capacity; and the unpruned cache 2*B*S*L*N*D*e with
+   * the same number of tokens. */
+  size_t model_think_bytes;
+  size_t model_dense_bytes;
+} thinK_sizes;
+
+typedef struct thinK_cache thinK_cache; /* opaque, host side */
+
+/* T = floor((1 - lambda) * D) (Sec. 3.1); returns 0 when lambda is outside
+ * [0, 1) or T would be 0. */
+int32_t thinK_T(double lambda, int32_t D);
+
+const char* thinK_status_string(thinK_status s);
+
+/* Sizes of the buffers thinK_create needs.  `seq_lens` (host, [B]) are the
+ * prompt lengths S_b; S_recent <= S_b, S_obs <= S_b <= S_max.
+ *
+ * Library layout of k_thin: for every (b, l, h) the S_p = S_b - S_recent prefix
+ * tokens are cut into tiles of 64 tokens; a tile is stored channel-major,
+ * [T][64] elements, rows of 64 tokens whose 16-byte chunks are XOR-swizzled with
+ * (row & 7) so that one bulk copy lands it in shared memory bank-conflict free.
+ * Logical element (token t, kept channel c) of head (b, l, h) sits at element
+ *   ((thin_tile_base(b) + (l*N_kv + h)*n_tiles(b) + t/64) * T + c) * 64 + swz(c, t%64)
+ * with n_tiles(b) = ceil(S_p(b)/64), thin_tile_base(b) = sum_{b'<b} L*N_kv*n_tiles(b'),
+ * swz(c, u) = (((u*e/16) ^ (c & 7)) * 16 + (u*e)%16) / e,  e = bytes/element.
+ * tail_k uses the same tile layout with all D channels: [B, L, N_kv, ceil(cap/64)][D][64],
+ * cap = S_recent + max_new_tokens. */
+thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens, thinK_sizes* out);
+
+/* Builds the host-side handle and writes the small device tables (lengths,
+ * tile offsets, zeroed counters) into `workspace` with synchronous copies.
+ * The buffers must be at least as large as thinK_cache_bytes reported and stay
+ * valid until thinK_destroy.  `scores` may be NULL (scores are then not kept). */
+thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void* k_thin, void* tail_k,
+                          void* tail_v, void* idx, void* scores, void* workspace, thinK_cache** out);
+
+/* Prefill, Sec. 3.2: channel scores and I = Top_T(Score, T) for layers
+ * [layer0, layer0 + nlayers) of every (b, h).
+ *   q_obs: [B, S_obs, L, N_q, D] view -- row s of entry b is the query of prompt
+ *          token S_b - S_obs + s ("Observation Window"); ignored (may hold a NULL
+ *          ptr) for the key-norm criteria of Eq. 1.
+ *   k:     [B, S_max, L, N_kv, D] view; rows >= S_b are never read.
+ * Score[j] = sqrt(sum_g sum_s q^2 * sum_t k^2): the closed form of the Frobenius
+ * norm of the rank-one product, with the G query heads of a group stacked.  All
+ * S_b key rows enter the score.  Sums run in fp64 over fp32 partial chains of
+ * at most 8 terms (bf16) or directly in fp64 (fp32), in a fixed order: results
+ * are deterministic.  Equal scores go to the lower channel.  Writes idx (and
+ * scores).  Layer indices address both the views and the cache. */
+thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, int32_t layer0,
+                                int32_t nlayers, void* stream);
+
+/* Prefill, Sec. 3.3: builds the two-part key cache for the given layers from
+ * the idx thinK_score_select stored: K_T[t][c] = K[t][idx[c]] for t < S_p, and
+ * the last S_recent rows of K and V copied unpruned to the tail.  After this
+ * call K may be released by the caller; V rows [0, S_p) of `v` stay BORROWED:
+ * thinK_decode_attn reads them in place on every step. */
+thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0, int32_t nlayers,
+                           void* stream);
+
+/* Decode, Sec. 3.3: the new token's key and value join the unpruned tail.
+ * k_new, v_new: dense [B, nlayers, N_kv, D].  Every layer of the cache must be
+ * appended once per step (any split into layer ranges); THINK_ERR_CAPACITY once
+ * max_new_tokens have been appended. */
+thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, int32_t layer0, int32_t nlayers,
+                          void* stream);
+
+/* Decode, Sec. 3.3 / Fig. 2 with the attention of Sec. 3.2: for each query head
+ * the query is gathered to the kept channels and multiplied with the pruned
+ * keys, the full query with the unpruned tail keys; the logits are concatenated,
+ * scaled by 1/sqrt(D) (original D) and normalised by ONE softmax; the result is
+ * the weighted sum of all value rows (prompt V in place + tail).
+ *   q, out: dense [B, nlayers, N_q, D] in the cache dtype.
+ * bf16: fp32 accumulation; fp32: logits in fp64, fp32 accumulation of p.V.
+ * All layers in the range must hold the same number of tail tokens. */
+thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
+                               void* stream);
+
+/* Tokens currently in the unpruned tail of `layer` (S_recent + appended), or -1. */
+int32_t thinK_tail_len(const thinK_cache* c, int32_t layer);
+
+/* Reads the device-side error word (0 = none) with a synchronous copy. */
+thinK_status thinK_device_error(thinK_cache* c, int32_t* out_code);
+
+thinK_status thinK_destroy(thinK_cache* c);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* THINK_H_ */

@@ -1,0 +1,130 @@
+// Key-cache compaction (paper Sec. 3.3): K_T[t][c] = K[t][idx[c]] for the pruned prefix, written
+// as channel-major 64-token tiles ([T][64], 16-byte chunks XOR-swizzled by row), plus the writer
+// of the unpruned tail (recent prompt rows at prefill, the new token at decode).
+#include "think_internal.h"
+
+namespace think {
+namespace {
+
+// One CTA builds one tile: 64 token rows of one head are staged in shared memory (padded pitch),
+// every thread then gathers 16 bytes' worth of tokens of one kept channel, and the finished tile
+// image leaves with coalesced 16-byte stores.
+template <typename Tin>
+__global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
+  constexpr int E = sizeof(Tin);
+  constexpr int CH = 16 / E;             // elements per 16-byte chunk
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int D = p.D, T = p.T;
+  const int pitch = D * E + 16;          // bytes; odd number of 16-byte chunks per row
+  unsigned char* s_in = smem;                                   // [64][pitch]
+  unsigned char* s_out = smem + kTileTokens * pitch;            // [T][64*E]
+  uint8_t* s_idx = (uint8_t*)(s_out + T * kTileTokens * E);     // [T]
+
+  const int tile = blockIdx.x, h = blockIdx.y;
+  const int b = blockIdx.z / p.nlayers, l = p.layer0 + blockIdx.z % p.nlayers;
+  const int S_p = p.seq_len[b] - p.R;
+  const int ntiles = (S_p + kTileTokens - 1) / kTileTokens;
+  if (tile >= ntiles) return;
+  const int tok0 = tile * kTileTokens;
+  const int nvalid = min(kTileTokens, S_p - tok0);
+  const int tid = threadIdx.x;
+
+  const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+  for (int c = tid; c < T; c += blockDim.x) s_idx[c] = p.idx[unit * T + c];
+
+  const Tin* src = (const Tin*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn;
+  const int cpr = D / CH;                // chunks per row
+  for (int i = tid; i < kTileTokens * cpr; i += blockDim.x) {
+    int r = i / cpr, ck = i % cpr;
+    uint4 v = make_uint4(0, 0, 0, 0);    // rows past the prefix become zeros
+    if (r < nvalid) v = __ldg((const uint4*)(src + (int64_t)(tok0 + r) * p.k.ss + ck * CH));
+    *(uint4*)(s_in + r * pitch + ck * 16) = v;
+  }
+  __syncthreads();
+
+  // item (j, c): tokens [j*CH, (j+1)*CH) of kept channel c; consecutive lanes take consecutive c
+  const int nj = kTileTokens / CH;
+  for (int item = tid; item < nj * T; item += blockDim.x) {
+    int j = item / T, c = item % T;
+    int ch = s_idx[c];
+    __align__(16) Tin tmp[CH];
+#pragma unroll
+    for (int i = 0; i < CH; ++i) tmp[i] = *(const Tin*)(s_in + (j * CH + i) * pitch + ch * E);
+    *(uint4*)(s_out + c * kTileTokens * E + ((j ^ (c & 7)) << 4)) = *(const uint4*)tmp;
+  }
+  __syncthreads();
+
+  const int64_t gtile = p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * ntiles + tile;
+  uint4* dst = (uint4*)((unsigned char*)p.k_thin + gtile * T * kTileTokens * E);
+  const int n16 = T * kTileTokens * E / 16;
+  for (int i = tid; i < n16; i += blockDim.x) dst[i] = ((const uint4*)s_out)[i];
+}
+
+// Rows of unpruned keys and their values into the tail.  One thread moves one 16-byte chunk of
+// one row: the value chunk is copied as is, the key chunk is scattered into the channel-major tile.
+template <typename Tin>
+__global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
+  constexpr int E = sizeof(Tin);
+  constexpr int CH = 16 / E;
+  const int cpr = p.D / CH;
+  const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.nrows * cpr;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int ck = i % cpr;
+    int64_t r1 = i / cpr;
+    int r = r1 % p.nrows; r1 /= p.nrows;
+    int h = r1 % p.N_kv; r1 /= p.N_kv;
+    int ll = r1 % p.nlayers;
+    int b = r1 / p.nlayers;
+    int l = p.layer0 + ll;
+    int64_t srow = p.rows_from_seq_len ? (p.seq_len[b] - p.R + r) : r;
+    int sl = l - p.src_layer_base;
+    const Tin* ks = (const Tin*)p.k.ptr + b * p.k.sb + srow * p.k.ss + (int64_t)sl * p.k.sl + (int64_t)h * p.k.sn + ck * CH;
+    const Tin* vs = (const Tin*)p.v.ptr + b * p.v.sb + srow * p.v.ss + (int64_t)sl * p.v.sl + (int64_t)h * p.v.sn + ck * CH;
+    uint4 kv = __ldg((const uint4*)ks);
+    uint4 vv = __ldg((const uint4*)vs);
+    const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+    const int u = p.pos0 + r;                       // position in the tail
+    *(uint4*)((Tin*)p.tail_v + (unit * p.cap + u) * p.D + ck * CH) = vv;
+    unsigned char* tile = (unsigned char*)p.tail_k + (unit * p.tail_tiles_cap + u / kTileTokens) * (int64_t)p.D * kTileTokens * E;
+    const Tin* kk = (const Tin*)&kv;
+    const int uu = u % kTileTokens;
+#pragma unroll
+    for (int j = 0; j < CH; ++j) {
+      int c = ck * CH + j;
+      *(Tin*)(tile + c * kTileTokens * E + tile_swz_bytes(c, uu, E)) = kk[j];
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s) {
+  if (max_tiles <= 0) return cudaSuccess;
+  dim3 grid(max_tiles, p.N_kv, p.B * p.nlayers);
+  const int E = dtype == THINK_BF16 ? 2 : 4;
+  size_t smem = (size_t)kTileTokens * (p.D * E + 16) + (size_t)p.T * kTileTokens * E + ((p.T + 15) & ~15);
+  cudaError_t e;
+  if (dtype == THINK_BF16) {
+    e = cudaFuncSetAttribute(k_compact<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_compact<__nv_bfloat16><<<grid, 128, smem, s>>>(p);
+  } else {
+    e = cudaFuncSetAttribute(k_compact<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_compact<float><<<grid, 128, smem, s>>>(p);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s) {
+  const int E = dtype == THINK_BF16 ? 2 : 4;
+  const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.nrows * (p.D * E / 16);
+  if (total <= 0) return cudaSuccess;
+  int blocks = (int)((total + 255) / 256);
+  if (blocks > kSMs * 16) blocks = kSMs * 16;
+  if (dtype == THINK_BF16) k_tail_write<__nv_bfloat16><<<blocks, 256, 0, s>>>(p);
+  else k_tail_write<float><<<blocks, 256, 0, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace think

@@ -1,0 +1,219 @@
+// Channel scores and top-T selection (paper Sec. 3.2; Eq. 1 for the key-norm criteria).
+//
+// Score[j] = ||Q_obs[:, j] K[:, j]^T||_F = sqrt(sum q^2 * sum k^2): one streaming pass over K
+// accumulates per-channel energies.  A CTA owns (entry b, layer l, block of columns, token
+// range); a thread owns one 16-byte column chunk and walks the token range with independent
+// 16-byte loads.  bf16 squares are exact in fp32; fp32 chains of 8 terms are flushed into fp64.
+// The CTA that arrives last for its (b, l, column block) -- an atomic ticket, nobody waits --
+// adds the partials in split order (deterministic), forms the scores and ranks each head.
+#include "think_internal.h"
+
+namespace think {
+namespace {
+
+template <typename Tin>
+struct Chunk;
+template <>
+struct Chunk<__nv_bfloat16> {
+  static constexpr int CH = 8;
+  __device__ static void unpack(const uint4& v, float (&x)[8]) {
+    x[0] = bf16lo(v.x); x[1] = bf16hi(v.x); x[2] = bf16lo(v.y); x[3] = bf16hi(v.y);
+    x[4] = bf16lo(v.z); x[5] = bf16hi(v.z); x[6] = bf16lo(v.w); x[7] = bf16hi(v.w);
+  }
+};
+template <>
+struct Chunk<float> {
+  static constexpr int CH = 4;
+  __device__ static void unpack(const uint4& v, float (&x)[4]) {
+    x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
+    x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+  }
+};
+
+__device__ __forceinline__ uint4 ldg16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+// Rank-count selection of one head by one warp: channel j is kept when fewer than T channels
+// beat it, where k beats j if s[k] > s[j] or (s[k] == s[j] and k < j).  Output ascending.
+__device__ void select_head(const double* s, int D, int T, uint8_t* out, int lane) {
+  int base = 0;
+  for (int j0 = 0; j0 < D; j0 += 32) {
+    int j = j0 + lane;
+    bool keep = false;
+    if (j < D) {
+      double sj = s[j];
+      int rank = 0;
+      for (int k = 0; k < D; ++k) {
+        double sk = s[k];
+        rank += (sk > sj) || (sk == sj && k < j);
+      }
+      keep = rank < T;
+    }
+    unsigned m = __ballot_sync(0xffffffffu, keep);
+    if (keep) out[base + __popc(m & ((1u << lane) - 1u))] = (uint8_t)j;
+    base += __popc(m);
+  }
+}
+
+template <typename Tin, bool L1>
+__global__ void __launch_bounds__(kScoreThreads) k_colnorm_score_select(const ScoreParams p) {
+  constexpr int CH = Chunk<Tin>::CH;
+  constexpr bool kBf16 = sizeof(Tin) == 2;
+  __shared__ double red[kScoreThreads * CH];   // reused: row-lane reduction, then scores
+  __shared__ int s_last;
+
+  const int tid = threadIdx.x;
+  const int split = blockIdx.x, colblk = blockIdx.y, z = blockIdx.z;
+  const int b = z / p.nlayers, l = p.layer0 + z % p.nlayers;
+  const int cl = tid % p.CB, rl = tid / p.CB;
+  const int chunk = colblk * p.CB + cl;
+  const bool active = rl < p.RP && chunk < p.NC;
+  const int CPH = p.D / CH;
+  const int h = chunk / CPH, j0 = (chunk % CPH) * CH;
+  const int S_b = p.seq_len[b];
+  const int per = (S_b + p.nsplit - 1) / p.nsplit;
+  const int t0 = split * per;
+  const int t1 = min(S_b, t0 + per);
+
+  double kacc[CH], qacc[CH];
+#pragma unroll
+  for (int i = 0; i < CH; ++i) kacc[i] = 0.0, qacc[i] = 0.0;
+
+  if (active) {
+    const Tin* kb = (const Tin*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn + j0;
+    int t = t0 + rl;
+    const int step = p.RP;
+    constexpr int U = 8;
+    for (; t + (U - 1) * step < t1; t += U * step) {
+      uint4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) v[u] = ldg16(kb + (int64_t)(t + u * step) * p.k.ss);
+      if (kBf16) {
+        float part[CH];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) part[i] = 0.f;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          float x[CH];
+          Chunk<Tin>::unpack(v[u], x);
+#pragma unroll
+          for (int i = 0; i < CH; ++i) part[i] = L1 ? part[i] + fabsf(x[i]) : fmaf(x[i], x[i], part[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < CH; ++i) kacc[i] += (double)part[i];
+      } else {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          float x[CH];
+          Chunk<Tin>::unpack(v[u], x);
+#pragma unroll
+          for (int i = 0; i < CH; ++i) {
+            double d = (double)x[i];
+            kacc[i] = L1 ? kacc[i] + fabs(d) : fma(d, d, kacc[i]);
+          }
+        }
+      }
+    }
+    for (; t < t1; t += step) {
+      uint4 v = ldg16(kb + (int64_t)t * p.k.ss);
+      float x[CH];
+      Chunk<Tin>::unpack(v, x);
+#pragma unroll
+      for (int i = 0; i < CH; ++i) {
+        double d = (double)x[i];
+        kacc[i] = L1 ? kacc[i] + fabs(d) : fma(d, d, kacc[i]);
+      }
+    }
+    if (p.criterion == THINK_SCORE_QUERY_DRIVEN) {
+      // the window rows of the G query heads that share key head h (stacked)
+      const Tin* qb = (const Tin*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl + j0;
+      const int nrows = p.S_obs * p.G;
+      for (int rr = split * p.RP + rl; rr < nrows; rr += p.nsplit * p.RP) {
+        int s = rr / p.G, g = rr % p.G;
+        uint4 v = ldg16(qb + (int64_t)s * p.q.ss + (int64_t)(h * p.G + g) * p.q.sn);
+        float x[CH];
+        Chunk<Tin>::unpack(v, x);
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          double d = (double)x[i];
+          qacc[i] = fma(d, d, qacc[i]);
+        }
+      }
+    }
+  }
+
+  // reduce over the row lanes of this CTA (fixed order), once for k and once for q
+  const int CBE = p.CB * CH;  // elements per column block
+  double* my = p.partials + ((int64_t)(z * p.ncolblk + colblk) * p.nsplit + split) * 2 * CBE;
+  for (int pass = 0; pass < 2; ++pass) {
+    double* acc = pass == 0 ? kacc : qacc;
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < CH; ++i) red[tid * CH + i] = acc[i];   // tid = rl * CB + cl when rl < RP
+    __syncthreads();
+    if (rl == 0) {
+#pragma unroll
+      for (int i = 0; i < CH; ++i) {
+        double s = 0.0;
+        for (int r = 0; r < p.RP; ++r) s += red[(r * p.CB + cl) * CH + i];
+        my[pass * CBE + cl * CH + i] = s;
+      }
+    }
+  }
+
+  // ticket: the last CTA of this (b, l, column block) finishes the job
+  __threadfence();
+  __syncthreads();
+  uint32_t* ctr = p.counters + (z * p.ncolblk + colblk);
+  if (tid == 0) s_last = (atomicAdd(ctr, 1u) == (uint32_t)(p.nsplit - 1));
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  const double* base = p.partials + (int64_t)(z * p.ncolblk + colblk) * p.nsplit * 2 * CBE;
+  const int ncols = min(CBE, (p.NC - colblk * p.CB) * CH);
+  for (int c = tid; c < ncols; c += kScoreThreads) {
+    double kn = 0.0, qn = 0.0;
+    for (int s = 0; s < p.nsplit; ++s) {
+      kn += __ldcg(base + (int64_t)s * 2 * CBE + c);
+      qn += __ldcg(base + (int64_t)s * 2 * CBE + CBE + c);
+    }
+    double sc;
+    if (p.criterion == THINK_SCORE_QUERY_DRIVEN) sc = sqrt(qn * kn);
+    else if (p.criterion == THINK_SCORE_KEY_L2) sc = sqrt(kn);
+    else sc = kn;
+    red[c] = sc;
+  }
+  __syncthreads();
+  const int heads = ncols / p.D;
+  const int h_first = colblk * p.CB * CH / p.D;
+  const int warp = tid >> 5, lane = tid & 31;
+  for (int hh = warp; hh < heads; hh += kScoreThreads / 32) {
+    const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h_first + hh;
+    select_head(red + hh * p.D, p.D, p.T, p.idx + unit * p.T, lane);
+    if (p.scores)
+      for (int j = lane; j < p.D; j += 32) p.scores[unit * p.D + j] = red[hh * p.D + j];
+  }
+  if (tid == 0) *ctr = 0u;  // ready for the next call
+}
+
+}  // namespace
+
+cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s) {
+  dim3 grid(p.nsplit, p.ncolblk, p.B * p.nlayers);
+  const bool l1 = p.criterion == THINK_SCORE_KEY_L1;
+  if (dtype == THINK_BF16) {
+    if (l1) k_colnorm_score_select<__nv_bfloat16, true><<<grid, kScoreThreads, 0, s>>>(p);
+    else k_colnorm_score_select<__nv_bfloat16, false><<<grid, kScoreThreads, 0, s>>>(p);
+  } else {
+    if (l1) k_colnorm_score_select<float, true><<<grid, kScoreThreads, 0, s>>>(p);
+    else k_colnorm_score_select<float, false><<<grid, kScoreThreads, 0, s>>>(p);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace think
