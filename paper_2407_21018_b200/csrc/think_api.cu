@@ -1,0 +1,358 @@
+// Host side of the C ABI: validation, buffer sizing, bookkeeping of the tail length, launches.
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "think_internal.h"
+
+using namespace think;
+
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {            // byte offsets inside the workspace
+  size_t seq_len, cum_thin, thin_tile_base, error, score_counters, decode_counters;
+  size_t score_partials, decode_records, total;
+  size_t header_bytes;     // everything before score_partials (initialised by thinK_create)
+};
+
+struct Geometry {
+  int B, L, N_q, N_kv, D, G, T, S_obs, R, max_new, cap, tail_tiles_cap, E, dtype, criterion;
+  int NC, CB, ncolblk, RPmax;
+  int64_t total_thin_tiles;    // over all (b, l, h)
+  int max_thin_tiles;          // per (l, h) over b
+  std::vector<int32_t> seq_len, cum_thin;
+  std::vector<int64_t> thin_tile_base;
+};
+
+thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geometry* g) {
+  if (!c || !seq_lens) return THINK_ERR_INVALID_ARG;
+  if (c->B < 1 || c->L < 1 || c->N_q < 1 || c->N_kv < 1 || c->S_obs < 1 || c->S_recent < 0 ||
+      c->max_new_tokens < 0 || c->S_max < 1)
+    return THINK_ERR_INVALID_ARG;
+  if (c->N_q % c->N_kv != 0) return THINK_ERR_INVALID_ARG;
+  if (c->dtype != THINK_BF16 && c->dtype != THINK_F32) return THINK_ERR_UNSUPPORTED;
+  if (c->criterion < THINK_SCORE_QUERY_DRIVEN || c->criterion > THINK_SCORE_KEY_L1) return THINK_ERR_INVALID_ARG;
+  if (!decode_supported(c->dtype, c->D, c->N_q / c->N_kv)) return THINK_ERR_UNSUPPORTED;
+  const int T = thinK_T(c->lambda, c->D);
+  if (T < 1) return THINK_ERR_INVALID_ARG;
+  if ((int64_t)c->B * c->L > 65535) return THINK_ERR_UNSUPPORTED;
+  g->B = c->B; g->L = c->L; g->N_q = c->N_q; g->N_kv = c->N_kv; g->D = c->D; g->G = c->N_q / c->N_kv;
+  g->T = T; g->S_obs = c->S_obs; g->R = c->S_recent; g->max_new = c->max_new_tokens; g->cap = c->S_recent + c->max_new_tokens;
+  if (g->cap < 1) g->cap = 1;
+  g->tail_tiles_cap = (g->cap + kTileTokens - 1) / kTileTokens;
+  g->dtype = c->dtype; g->E = c->dtype == THINK_BF16 ? 2 : 4; g->criterion = c->criterion;
+  const int CH = 16 / g->E;
+  g->NC = c->N_kv * c->D / CH;
+  g->CB = g->NC < kScoreThreads ? g->NC : kScoreThreads;
+  g->ncolblk = (g->NC + g->CB - 1) / g->CB;
+  g->RPmax = kScoreThreads / g->CB;
+  g->seq_len.assign(seq_lens, seq_lens + c->B);
+  g->cum_thin.assign(c->B + 1, 0);
+  g->thin_tile_base.assign(c->B + 1, 0);
+  g->max_thin_tiles = 0;
+  for (int b = 0; b < c->B; ++b) {
+    const int S = seq_lens[b];
+    if (S < c->S_obs || S < c->S_recent || S > c->S_max || S < 1) return THINK_ERR_INVALID_ARG;
+    const int nt = (S - c->S_recent + kTileTokens - 1) / kTileTokens;
+    g->cum_thin[b + 1] = g->cum_thin[b] + nt;
+    g->thin_tile_base[b + 1] = g->thin_tile_base[b] + (int64_t)c->L * c->N_kv * nt;
+    if (nt > g->max_thin_tiles) g->max_thin_tiles = nt;
+  }
+  g->total_thin_tiles = g->thin_tile_base[c->B];
+  return THINK_OK;
+}
+
+void make_layout(const Geometry& g, Layout* w) {
+  size_t o = 0;
+  w->seq_len = o;          o = align_up(o + sizeof(int32_t) * g.B, 256);
+  w->cum_thin = o;         o = align_up(o + sizeof(int32_t) * (g.B + 1), 256);
+  w->thin_tile_base = o;   o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
+  w->error = o;            o = align_up(o + 256, 256);
+  w->score_counters = o;   o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.ncolblk, 256);
+  w->decode_counters = o;  o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.N_kv, 256);
+  w->header_bytes = o;
+  w->score_partials = o;
+  // a call splits tokens so that items * nsplit <= target + items
+  const size_t slots = (size_t)kScoreTargetCtas + (size_t)g.B * g.L * g.ncolblk;
+  o = align_up(o + slots * 2 * (size_t)g.CB * (16 / g.E) * sizeof(double), 256);
+  w->decode_records = o;
+  o = align_up(o + (size_t)kMaxDecodeCtas * 2 * decode_record_bytes(g.D, g.G), 256);
+  w->total = o;
+}
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+bool check_view(const thinK_tensor5& t, int E) {
+  if (!t.ptr || !aligned16(t.ptr)) return false;
+  const int64_t s[4] = {t.stride_b, t.stride_s, t.stride_l, t.stride_n};
+  for (int i = 0; i < 4; ++i)
+    if (s[i] < 0 || (s[i] * E) % 16 != 0) return false;
+  return true;
+}
+
+View5 to_view(const thinK_tensor5& t) { return View5{t.ptr, t.stride_b, t.stride_s, t.stride_l, t.stride_n}; }
+
+}  // namespace
+
+struct thinK_cache {
+  Geometry g;
+  Layout w;
+  unsigned char* ws;
+  void *k_thin, *tail_k, *tail_v, *idx, *scores;
+  std::vector<uint8_t> scored, compacted;   // per layer
+  std::vector<int32_t> tail_len;            // per layer, tokens in the tail
+  thinK_tensor5 v;                          // borrowed prompt values (set by thinK_compact)
+  bool have_v;
+  int num_sms, decode_grid_max;
+};
+
+extern "C" {
+
+int32_t thinK_T(double lambda, int32_t D) {
+  if (!(lambda >= 0.0 && lambda < 1.0) || D < 1) return 0;
+  const int32_t T = (int32_t)floor((1.0 - lambda) * (double)D + 1e-9);
+  return T < 1 ? 0 : (T > D ? D : T);
+}
+
+const char* thinK_status_string(thinK_status s) {
+  switch (s) {
+    case THINK_OK: return "ok";
+    case THINK_ERR_INVALID_ARG: return "invalid argument";
+    case THINK_ERR_UNSUPPORTED: return "unsupported configuration";
+    case THINK_ERR_STATE: return "call out of order";
+    case THINK_ERR_CAPACITY: return "capacity exceeded";
+    case THINK_ERR_CUDA: return "CUDA error";
+  }
+  return "unknown status";
+}
+
+thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens, thinK_sizes* out) {
+  if (!out) return THINK_ERR_INVALID_ARG;
+  Geometry g;
+  thinK_status st = make_geometry(cfg, seq_lens, &g);
+  if (st != THINK_OK) return st;
+  Layout w;
+  make_layout(g, &w);
+  const size_t units = (size_t)g.B * g.L * g.N_kv;
+  out->k_thin = align_up((size_t)g.total_thin_tiles * g.T * kTileTokens * g.E, 256);
+  if (out->k_thin == 0) out->k_thin = 256;
+  out->tail_k = align_up(units * g.tail_tiles_cap * (size_t)g.D * kTileTokens * g.E, 256);
+  out->tail_v = align_up(units * g.cap * (size_t)g.D * g.E, 256);
+  out->idx = align_up(units * g.T, 256);
+  out->scores = align_up(units * g.D * sizeof(double), 256);
+  out->workspace = w.total;
+  size_t think_elems = 0, dense_elems = 0;
+  const int new_tokens = cfg->max_new_tokens;
+  for (int b = 0; b < g.B; ++b) {
+    const size_t S = g.seq_len[b], S_p = S - g.R;
+    think_elems += S_p * g.T + (size_t)(g.R + new_tokens) * g.D + (S + new_tokens) * g.D;
+    dense_elems += 2 * (S + new_tokens) * g.D;
+  }
+  out->model_think_bytes = think_elems * g.L * g.N_kv * g.E;
+  out->model_dense_bytes = dense_elems * g.L * g.N_kv * g.E;
+  return THINK_OK;
+}
+
+thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void* k_thin, void* tail_k,
+                          void* tail_v, void* idx, void* scores, void* workspace, thinK_cache** out) {
+  if (!out) return THINK_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!k_thin || !tail_k || !tail_v || !idx || !workspace) return THINK_ERR_INVALID_ARG;
+  if (!aligned16(k_thin) || !aligned16(tail_k) || !aligned16(tail_v) || !aligned16(workspace) ||
+      (scores && !aligned16(scores)))
+    return THINK_ERR_INVALID_ARG;
+  thinK_cache* c = new (std::nothrow) thinK_cache();
+  if (!c) return THINK_ERR_INVALID_ARG;
+  thinK_status st = make_geometry(cfg, seq_lens, &c->g);
+  if (st != THINK_OK) { delete c; return st; }
+  make_layout(c->g, &c->w);
+  c->ws = (unsigned char*)workspace;
+  c->k_thin = k_thin; c->tail_k = tail_k; c->tail_v = tail_v; c->idx = idx; c->scores = scores;
+  c->scored.assign(c->g.L, 0);
+  c->compacted.assign(c->g.L, 0);
+  c->tail_len.assign(c->g.L, 0);
+  c->have_v = false;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    delete c;
+    return THINK_ERR_CUDA;
+  }
+  c->num_sms = prop.multiProcessorCount;
+  int occ = decode_ctas_per_sm(c->g.dtype, c->g.D, c->g.G);
+  if (occ < 1) { delete c; return THINK_ERR_CUDA; }
+  c->decode_grid_max = c->num_sms * occ;
+  if (c->decode_grid_max > kMaxDecodeCtas) c->decode_grid_max = kMaxDecodeCtas;
+  // device tables
+  const Geometry& g = c->g;
+  bool ok = cudaMemset(c->ws, 0, c->w.header_bytes) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->ws + c->w.seq_len, g.seq_len.data(), sizeof(int32_t) * g.B, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->ws + c->w.cum_thin, g.cum_thin.data(), sizeof(int32_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->ws + c->w.thin_tile_base, g.thin_tile_base.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
+  if (!ok) { delete c; return THINK_ERR_CUDA; }
+  *out = c;
+  return THINK_OK;
+}
+
+static bool layer_range_ok(const thinK_cache* c, int layer0, int nlayers) {
+  return layer0 >= 0 && nlayers >= 1 && layer0 + nlayers <= c->g.L;
+}
+
+thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, int32_t layer0,
+                                int32_t nlayers, void* stream) {
+  if (!c) return THINK_ERR_INVALID_ARG;
+  if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
+  const Geometry& g = c->g;
+  if (!check_view(k, g.E)) return THINK_ERR_INVALID_ARG;
+  if (g.criterion == THINK_SCORE_QUERY_DRIVEN && !check_view(q_obs, g.E)) return THINK_ERR_INVALID_ARG;
+  ScoreParams p;
+  memset(&p, 0, sizeof(p));
+  p.k = to_view(k);
+  p.q = to_view(q_obs);
+  p.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
+  p.partials = (double*)(c->ws + c->w.score_partials);
+  p.counters = (uint32_t*)(c->ws + c->w.score_counters);
+  p.idx = (uint8_t*)c->idx;
+  p.scores = (double*)c->scores;
+  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.G = g.G; p.D = g.D; p.T = g.T; p.S_obs = g.S_obs;
+  p.layer0 = layer0; p.nlayers = nlayers;
+  p.NC = g.NC; p.CB = g.CB; p.ncolblk = g.ncolblk; p.RP = g.RPmax;
+  p.criterion = g.criterion;
+  const int items = g.B * nlayers * g.ncolblk;
+  int nsplit = (kScoreTargetCtas + items - 1) / items;
+  // keep at least 64 token rows per row lane of a split
+  int min_len = g.seq_len[0];
+  for (int b = 1; b < g.B; ++b) min_len = g.seq_len[b] < min_len ? g.seq_len[b] : min_len;
+  int cap = min_len / (64 * p.RP);
+  if (cap < 1) cap = 1;
+  if (nsplit > cap) nsplit = cap;
+  if (nsplit < 1) nsplit = 1;
+  p.nsplit = nsplit;
+  if (launch_score(p, g.dtype, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  for (int l = layer0; l < layer0 + nlayers; ++l) c->scored[l] = 1;
+  return THINK_OK;
+}
+
+thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0, int32_t nlayers,
+                           void* stream) {
+  if (!c) return THINK_ERR_INVALID_ARG;
+  if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
+  const Geometry& g = c->g;
+  if (!check_view(k, g.E) || !check_view(v, g.E)) return THINK_ERR_INVALID_ARG;
+  for (int l = layer0; l < layer0 + nlayers; ++l)
+    if (!c->scored[l]) return THINK_ERR_STATE;
+  if (c->have_v && memcmp(&c->v, &v, sizeof(v)) != 0) return THINK_ERR_INVALID_ARG;  // one V for all layers
+  CompactParams p;
+  memset(&p, 0, sizeof(p));
+  p.k = to_view(k);
+  p.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
+  p.thin_tile_base = (const int64_t*)(c->ws + c->w.thin_tile_base);
+  p.idx = (const uint8_t*)c->idx;
+  p.k_thin = c->k_thin;
+  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.D = g.D; p.T = g.T; p.R = g.R;
+  p.layer0 = layer0; p.nlayers = nlayers;
+  if (launch_compact(p, g.dtype, g.max_thin_tiles, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  if (g.R > 0) {
+    TailWriteParams t;
+    memset(&t, 0, sizeof(t));
+    t.k = to_view(k); t.v = to_view(v);
+    t.src_layer_base = 0; t.rows_from_seq_len = 1;
+    t.seq_len = p.seq_len;
+    t.tail_k = c->tail_k; t.tail_v = c->tail_v;
+    t.B = g.B; t.L = g.L; t.N_kv = g.N_kv; t.D = g.D; t.R = g.R; t.cap = g.cap; t.tail_tiles_cap = g.tail_tiles_cap;
+    t.layer0 = layer0; t.nlayers = nlayers; t.nrows = g.R; t.pos0 = 0;
+    if (launch_tail_write(t, g.dtype, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  }
+  c->v = v;
+  c->have_v = true;
+  for (int l = layer0; l < layer0 + nlayers; ++l) { c->compacted[l] = 1; c->tail_len[l] = g.R; }
+  return THINK_OK;
+}
+
+thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, int32_t layer0, int32_t nlayers,
+                          void* stream) {
+  if (!c || !k_new || !v_new) return THINK_ERR_INVALID_ARG;
+  if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new)) return THINK_ERR_INVALID_ARG;
+  const Geometry& g = c->g;
+  const int pos = c->tail_len[layer0];
+  for (int l = layer0; l < layer0 + nlayers; ++l) {
+    if (!c->compacted[l]) return THINK_ERR_STATE;
+    if (c->tail_len[l] != pos) return THINK_ERR_STATE;
+  }
+  if (pos - g.R >= g.max_new || pos >= g.cap) return THINK_ERR_CAPACITY;
+  TailWriteParams t;
+  memset(&t, 0, sizeof(t));
+  const int64_t sn = g.D, sl = (int64_t)g.N_kv * g.D, sb = (int64_t)nlayers * sl;
+  t.k = View5{k_new, sb, 0, sl, sn};
+  t.v = View5{v_new, sb, 0, sl, sn};
+  t.src_layer_base = layer0; t.rows_from_seq_len = 0;
+  t.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
+  t.tail_k = c->tail_k; t.tail_v = c->tail_v;
+  t.B = g.B; t.L = g.L; t.N_kv = g.N_kv; t.D = g.D; t.R = g.R; t.cap = g.cap; t.tail_tiles_cap = g.tail_tiles_cap;
+  t.layer0 = layer0; t.nlayers = nlayers; t.nrows = 1; t.pos0 = pos;
+  if (launch_tail_write(t, g.dtype, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  for (int l = layer0; l < layer0 + nlayers; ++l) c->tail_len[l] = pos + 1;
+  return THINK_OK;
+}
+
+thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
+                               void* stream) {
+  if (!c || !q || !out) return THINK_ERR_INVALID_ARG;
+  if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return THINK_ERR_INVALID_ARG;
+  const Geometry& g = c->g;
+  const int n_tail = c->tail_len[layer0];
+  for (int l = layer0; l < layer0 + nlayers; ++l) {
+    if (!c->compacted[l]) return THINK_ERR_STATE;
+    if (c->tail_len[l] != n_tail) return THINK_ERR_STATE;
+  }
+  DecodeParams p;
+  memset(&p, 0, sizeof(p));
+  p.k_thin = c->k_thin; p.tail_k = c->tail_k; p.tail_v = c->tail_v;
+  p.v = to_view(c->v);
+  p.idx = (const uint8_t*)c->idx;
+  p.q = q; p.out = out;
+  p.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
+  p.cum_thin = (const int32_t*)(c->ws + c->w.cum_thin);
+  p.thin_tile_base = (const int64_t*)(c->ws + c->w.thin_tile_base);
+  p.records = c->ws + c->w.decode_records;
+  p.counters = (uint32_t*)(c->ws + c->w.decode_counters);
+  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.N_q = g.N_q; p.T = g.T; p.R = g.R; p.cap = g.cap;
+  p.tail_tiles_cap = g.tail_tiles_cap;
+  p.n_tail = n_tail;
+  p.n_tail_tiles = (n_tail + kTileTokens - 1) / kTileTokens;
+  p.layer0 = layer0; p.nlayers = nlayers;
+  p.Ntot = (long long)nlayers * g.N_kv * ((long long)g.cum_thin[g.B] + (long long)g.B * p.n_tail_tiles);
+  for (int b = 0; b < g.B; ++b)
+    if (g.cum_thin[b + 1] - g.cum_thin[b] + p.n_tail_tiles < 1) return THINK_ERR_STATE;  // nothing to attend to
+  p.grid = (int)(p.Ntot < (long long)c->decode_grid_max ? p.Ntot : (long long)c->decode_grid_max);
+  if (launch_decode(p, g.dtype, g.D, g.G, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  return THINK_OK;
+}
+
+int32_t thinK_tail_len(const thinK_cache* c, int32_t layer) {
+  if (!c || layer < 0 || layer >= c->g.L) return -1;
+  return c->tail_len[layer];
+}
+
+thinK_status thinK_device_error(thinK_cache* c, int32_t* out_code) {
+  if (!c || !out_code) return THINK_ERR_INVALID_ARG;
+  uint32_t v = 0;
+  if (cudaMemcpy(&v, c->ws + c->w.error, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) return THINK_ERR_CUDA;
+  *out_code = (int32_t)v;
+  return THINK_OK;
+}
+
+thinK_status thinK_destroy(thinK_cache* c) {
+  if (!c) return THINK_ERR_INVALID_ARG;
+  delete c;
+  return THINK_OK;
+}
+
+}  // extern "C"
