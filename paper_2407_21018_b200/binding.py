@@ -1,0 +1,249 @@
+"""ctypes binding of libthink.so -- argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; this module turns
+torch tensors into pointers/strides, allocates the caller-owned buffers with
+``torch.empty`` and forwards the current CUDA stream.  Importing it raises if
+the compiled library is missing: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libthink.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} not found: build it first (python -m paper_2407_21018_b200.build); "
+        "the CUDA library is the only implementation of this path")
+
+lib = C.CDLL(LIB_PATH)
+
+THINK_OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_STATE, ERR_CAPACITY, ERR_CUDA = range(6)
+BF16, F32 = 0, 1
+SCORE_QUERY_DRIVEN, SCORE_KEY_L2, SCORE_KEY_L1 = 0, 1, 2
+TILE_TOKENS = 64
+
+
+class Config(C.Structure):
+    _fields_ = [("B", C.c_int32), ("L", C.c_int32), ("N_q", C.c_int32), ("N_kv", C.c_int32), ("D", C.c_int32),
+                ("S_max", C.c_int32), ("S_obs", C.c_int32), ("S_recent", C.c_int32),
+                ("max_new_tokens", C.c_int32), ("dtype", C.c_int32), ("criterion", C.c_int32),
+                ("reserved", C.c_int32), ("lam", C.c_double)]
+
+
+class Tensor5(C.Structure):
+    _fields_ = [("ptr", C.c_void_p), ("stride_b", C.c_int64), ("stride_s", C.c_int64),
+                ("stride_l", C.c_int64), ("stride_n", C.c_int64)]
+
+
+class Sizes(C.Structure):
+    _fields_ = [("k_thin", C.c_size_t), ("tail_k", C.c_size_t), ("tail_v", C.c_size_t), ("idx", C.c_size_t),
+                ("scores", C.c_size_t), ("workspace", C.c_size_t), ("model_think_bytes", C.c_size_t),
+                ("model_dense_bytes", C.c_size_t)]
+
+
+EXPORTS = {
+    "thinK_T": (C.c_int32, [C.c_double, C.c_int32]),
+    "thinK_status_string": (C.c_char_p, [C.c_int]),
+    "thinK_cache_bytes": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32), C.POINTER(Sizes)]),
+    "thinK_create": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32)] + [C.c_void_p] * 6 + [C.POINTER(C.c_void_p)]),
+    "thinK_score_select": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_compact": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_append": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_decode_attn": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_tail_len": (C.c_int32, [C.c_void_p, C.c_int32]),
+    "thinK_device_error": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32)]),
+    "thinK_destroy": (C.c_int, [C.c_void_p]),
+}
+for _name, (_res, _args) in EXPORTS.items():
+    _fn = getattr(lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+
+class ThinKError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib.thinK_status_string(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str):
+    if status != THINK_OK:
+        raise ThinKError(status, where)
+
+
+def thinK_T(lam: float, D: int) -> int:
+    return int(lib.thinK_T(lam, D))
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.bfloat16:
+        return BF16
+    if dt == torch.float32:
+        return F32
+    raise ThinKError(ERR_UNSUPPORTED, "dtype")
+
+
+def tensor5(t: Optional[torch.Tensor]) -> Tensor5:
+    """View of a 5-d tensor indexed [b, s, l, n, d] with d contiguous (any strides otherwise)."""
+    if t is None:
+        return Tensor5(None, 0, 0, 0, 0)
+    assert t.dim() == 5 and t.stride(4) == 1
+    return Tensor5(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2), t.stride(3))
+
+
+def make_config(B, L, N_q, N_kv, D, S_max, S_obs, S_recent, max_new_tokens, lam, dtype, criterion=SCORE_QUERY_DRIVEN):
+    return Config(B, L, N_q, N_kv, D, S_max, S_obs, S_recent, max_new_tokens,
+                  dtype if isinstance(dtype, int) else _dtype_code(dtype), criterion, 0, float(lam))
+
+
+def thinK_cache_bytes(cfg: Config, seq_lens: Sequence[int]) -> Sizes:
+    arr = (C.c_int32 * len(seq_lens))(*seq_lens)
+    out = Sizes()
+    _check(lib.thinK_cache_bytes(C.byref(cfg), arr, C.byref(out)), "thinK_cache_bytes")
+    return out
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+class ThinKCache:
+    """Owns the caller-side buffers (torch allocations) and the library handle."""
+
+    def __init__(self, cfg: Config, seq_lens: Sequence[int], device="cuda", keep_scores: bool = True):
+        self.cfg = cfg
+        self.seq_lens = [int(s) for s in seq_lens]
+        self.sizes = thinK_cache_bytes(cfg, self.seq_lens)
+        self.device = torch.device(device)
+        self.T = thinK_T(cfg.lam, cfg.D)
+        self.torch_dtype = torch.bfloat16 if cfg.dtype == BF16 else torch.float32
+        self.elem = 2 if cfg.dtype == BF16 else 4
+        mk = lambda n: torch.empty(max(int(n), 256), dtype=torch.uint8, device=self.device)
+        self.k_thin = mk(self.sizes.k_thin)
+        self.tail_k = mk(self.sizes.tail_k)
+        self.tail_v = mk(self.sizes.tail_v)
+        self.idx = mk(self.sizes.idx)
+        self.scores = mk(self.sizes.scores) if keep_scores else None
+        self.workspace = mk(self.sizes.workspace)
+        self._v = None
+        arr = (C.c_int32 * len(self.seq_lens))(*self.seq_lens)
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(lib.thinK_create(C.byref(cfg), arr, self.k_thin.data_ptr(), self.tail_k.data_ptr(),
+                                    self.tail_v.data_ptr(), self.idx.data_ptr(),
+                                    self.scores.data_ptr() if self.scores is not None else None,
+                                    self.workspace.data_ptr(), C.byref(h)), "thinK_create")
+        self.handle = h
+
+    # -- the four calls of the path -------------------------------------
+    def score_select(self, q_obs: Optional[torch.Tensor], k: torch.Tensor, layer0=0, nlayers=None, stream=None):
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        _check(lib.thinK_score_select(self.handle, tensor5(q_obs), tensor5(k), layer0, nlayers, _stream_ptr(stream)),
+               "thinK_score_select")
+
+    def compact(self, k: torch.Tensor, v: torch.Tensor, layer0=0, nlayers=None, stream=None):
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        self._v = v   # borrowed by the library: keep it alive
+        _check(lib.thinK_compact(self.handle, tensor5(k), tensor5(v), layer0, nlayers, _stream_ptr(stream)),
+               "thinK_compact")
+
+    def append(self, k_new: torch.Tensor, v_new: torch.Tensor, layer0=0, nlayers=None, stream=None):
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        assert k_new.is_contiguous() and v_new.is_contiguous()
+        _check(lib.thinK_append(self.handle, k_new.data_ptr(), v_new.data_ptr(), layer0, nlayers, _stream_ptr(stream)),
+               "thinK_append")
+
+    def decode_attn(self, q: torch.Tensor, out: Optional[torch.Tensor] = None, layer0=0, nlayers=None, stream=None):
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        assert q.is_contiguous()
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib.thinK_decode_attn(self.handle, q.data_ptr(), out.data_ptr(), layer0, nlayers, _stream_ptr(stream)),
+               "thinK_decode_attn")
+        return out
+
+    # -- inspection ------------------------------------------------------
+    def tail_len(self, layer=0) -> int:
+        return int(lib.thinK_tail_len(self.handle, layer))
+
+    def device_error(self) -> int:
+        code = C.c_int32(0)
+        _check(lib.thinK_device_error(self.handle, C.byref(code)), "thinK_device_error")
+        return code.value
+
+    def idx_tensor(self) -> torch.Tensor:
+        c = self.cfg
+        n = c.B * c.L * c.N_kv * self.T
+        return self.idx[:n].view(c.B, c.L, c.N_kv, self.T)
+
+    def scores_tensor(self) -> torch.Tensor:
+        c = self.cfg
+        n = c.B * c.L * c.N_kv * c.D * 8
+        return self.scores[:n].view(torch.float64).view(c.B, c.L, c.N_kv, c.D)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib.thinK_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+# ---------------------------------------------------------------------------
+# Address arithmetic of the documented library layout (for readers of k_thin /
+# tail_k, e.g. tests): pure indexing, no arithmetic of the method.
+# ---------------------------------------------------------------------------
+def swz(c: int, u: int, e: int) -> int:
+    """Element offset of token u (0..63) in row c of a channel-major tile."""
+    byte = u * e
+    return ((((byte >> 4) ^ (c & 7)) << 4) | (byte & 15)) // e
+
+
+def unpack_tiles(raw: torch.Tensor, n_tiles: int, rows: int, n_tokens: int, dtype: torch.dtype) -> torch.Tensor:
+    """raw: flat tensor of `dtype` holding n_tiles tiles [rows][64] (swizzled);
+    returns the logical [n_tokens, rows] matrix."""
+    e = raw.element_size()
+    t = raw[: n_tiles * rows * TILE_TOKENS].view(n_tiles, rows, TILE_TOKENS)
+    c = torch.arange(rows, device=raw.device)[:, None]
+    u = torch.arange(TILE_TOKENS, device=raw.device)[None, :]
+    byte = u * e
+    off = ((((byte >> 4) ^ (c & 7)) << 4) | (byte & 15)) // e          # [rows, 64]
+    logical = torch.gather(t, 2, off[None].expand(n_tiles, -1, -1))    # [tile, row, u]
+    return logical.permute(0, 2, 1).reshape(n_tiles * TILE_TOKENS, rows)[:n_tokens]
+
+
+def k_thin_logical(cache: ThinKCache, b: int, l: int, h: int) -> torch.Tensor:
+    """Pruned prefix keys of one head as [S_p, T]."""
+    c = cache.cfg
+    S_p = cache.seq_lens[b] - c.S_recent
+    nt = [(s - c.S_recent + TILE_TOKENS - 1) // TILE_TOKENS for s in cache.seq_lens]
+    base = sum(c.L * c.N_kv * x for x in nt[:b]) + (l * c.N_kv + h) * nt[b]
+    flat = cache.k_thin.view(cache.torch_dtype)
+    per = cache.T * TILE_TOKENS
+    return unpack_tiles(flat[base * per:(base + nt[b]) * per], nt[b], cache.T, S_p, cache.torch_dtype)
+
+
+def tail_logical(cache: ThinKCache, b: int, l: int, h: int):
+    """Unpruned tail of one head: (keys [n, D], values [n, D])."""
+    c = cache.cfg
+    n = cache.tail_len(l)
+    cap = max(1, c.S_recent + c.max_new_tokens)
+    ttc = (cap + TILE_TOKENS - 1) // TILE_TOKENS
+    unit = (b * c.L + l) * c.N_kv + h
+    per = c.D * TILE_TOKENS
+    flat = cache.tail_k.view(cache.torch_dtype)
+    keys = unpack_tiles(flat[unit * ttc * per:(unit + 1) * ttc * per], ttc, c.D, n, cache.torch_dtype)
+    vals = cache.tail_v.view(cache.torch_dtype)[unit * cap * c.D:(unit * cap + n) * c.D].view(n, c.D)
+    return keys, vals

@@ -1,0 +1,269 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Selected indices and cache contents bit-exact; attention within
+1e-2 (bf16 I/O) / 1e-5 (fp32 I/O) max-abs."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import think_oracle as orc
+from paper_2407_21018_b200 import workloads as wl
+
+from _harness import (assert_attn_close, compare_cache, compare_selection, make_cache, make_oracle, run_case, to64)
+
+pytestmark = pytest.mark.gpu
+
+
+def test_c1_full():
+    """Config 1 exactly as stated: fp32, 4 MHA heads, D=64, S=512, 8 decode steps."""
+    r = run_case(wl.get_config("c1"))
+    assert r["max_abs"] <= 1e-5
+
+
+@pytest.mark.parametrize("name,S,L,B,steps", [
+    ("c2", 2048 + 37, 2, 1, 6),      # GQA 4:1, RoPE, ragged last tile
+    ("c3", 1500, 2, 2, 4),           # batch of equal lengths
+    ("c4", 700, 1, 5, 5),            # MHA, ragged batch, outlier channels, T = 51
+    ("c5", 3000, 1, 1, 70),          # S_obs = 64; tail grows past one 64-token tile
+])
+def test_shrunk_configs(name, S, L, B, steps):
+    w = wl.shrink(wl.get_config(name), S=S, L=L, B=B, steps=steps)
+    run_case(w)
+
+
+@pytest.mark.parametrize("lam", [0.0, 0.25, 0.75])
+def test_lambda_sweep(lam):
+    w = wl.shrink(wl.get_config("c5"), S=1000, L=1, steps=3, lam=lam)
+    run_case(w)
+
+
+def test_lambda_zero_is_dense_attention():
+    """lambda = 0 keeps every channel: the CUDA path must then equal plain dense attention."""
+    w = wl.shrink(wl.get_config("c2"), S=777, L=1, steps=2, lam=0.0)
+    r = run_case(w)
+    o = r["oracle"]
+    assert (o.idx == np.arange(w.D)).all()
+
+
+@pytest.mark.parametrize("R", [0, 1, 128])
+def test_recent_sizes(R):
+    w = dataclasses.replace(wl.shrink(wl.get_config("c2"), S=600, L=1, steps=3), S_recent=R)
+    run_case(w)
+
+
+def test_all_tokens_recent():
+    """S_recent = S: empty pruned prefix, everything lives in the unpruned tail."""
+    w = wl.shrink(wl.get_config("c1"), S=96, steps=3)
+    w = dataclasses.replace(w, S_recent=w.seq_lens[0])
+    run_case(w)
+
+
+def test_shortest_prompt():
+    """S = S_obs + 1 (one pruned token) and S = S_obs with S_recent = 0."""
+    w = wl.shrink(wl.get_config("c1"), S=33, steps=2)
+    run_case(w)
+    w = dataclasses.replace(wl.shrink(wl.get_config("c1"), S=33, steps=2), seq_lens=(32,), S_recent=0)
+    run_case(w)
+
+
+@pytest.mark.parametrize("dtype,D,G", [("f32", 128, 2), ("bf16", 64, 8), ("f32", 64, 1), ("bf16", 128, 1),
+                                       ("bf16", 64, 2), ("f32", 128, 4)])
+def test_shapes(dtype, D, G):
+    w = wl.Workload("shape", dtype, 2, 2, 2 * G, 2, D, (300, 171), 16, 0.4, 3, 10000.0, (2, 10.0), 0x5EED + D + G)
+    run_case(w)
+
+
+@pytest.mark.parametrize("criterion", [1, 2])
+def test_magnitude_criteria(criterion):
+    """Eq. 1 criteria (key l2 / l1 norms) through the same kernels."""
+    w = wl.shrink(wl.get_config("c4"), S=500, L=1, B=2, steps=2)
+    run_case(w, criterion=criterion)
+
+
+def test_exact_ties_go_to_lower_channel():
+    """Duplicate channels give exactly equal scores; the lower index must win on both sides."""
+    w = wl.shrink(wl.get_config("c1"), S=200, steps=0)
+    data = wl.make_prefill(w, device="cpu")
+    K, Q = data["K"], data["Q_obs"]
+    for a, b in ((3, 40), (7, 8), (10, 63)):
+        K[..., b] = K[..., a]
+        Q[..., b] = Q[..., a]
+    cache = make_cache(w, 0)
+    cache.score_select(Q.cuda(), K.cuda())
+    torch.cuda.synchronize()
+    o = make_oracle(w)
+    o.score_select(to64(Q), to64(K))
+    got = cache.idx_tensor().cpu().numpy().astype(np.int64)
+    assert (got == o.idx).all()
+    sc = cache.scores_tensor().cpu().numpy()
+    assert (sc[..., 3] == sc[..., 40]).all()
+
+
+def test_layer_ranges_and_determinism():
+    """Per-layer calls give the same bytes as one call over all layers, and a repeat is identical."""
+    w = wl.shrink(wl.get_config("c2"), S=900, L=3, steps=2)
+    data = wl.make_prefill(w, device="cpu")
+    K, V, Q = data["K"].cuda(), data["V"].cuda(), data["Q_obs"].cuda()
+    a, b = make_cache(w, 2), make_cache(w, 2)
+    a.score_select(Q, K)
+    a.compact(K, V)
+    for l in (2, 0, 1):
+        b.score_select(Q, K, layer0=l, nlayers=1)
+        b.compact(K, V, layer0=l, nlayers=1)
+    torch.cuda.synchronize()
+    assert torch.equal(a.idx_tensor(), b.idx_tensor())
+    n = a.sizes.k_thin
+    assert torch.equal(a.k_thin[:n], b.k_thin[:n])
+    st = wl.make_step(w, 0, device="cuda")
+    a.append(st["k_new"], st["v_new"])
+    out_a = a.decode_attn(st["q"])
+    out_a2 = a.decode_attn(st["q"])
+    outs = []
+    for l in range(3):
+        b.append(st["k_new"][:, l:l + 1].contiguous(), st["v_new"][:, l:l + 1].contiguous(), layer0=l, nlayers=1)
+        outs.append(b.decode_attn(st["q"][:, l:l + 1].contiguous(), layer0=l, nlayers=1))
+    torch.cuda.synchronize()
+    assert torch.equal(out_a, out_a2)
+    got = torch.cat(outs, dim=1)
+    # split boundaries differ between the two launch shapes: same values up to fp32 merge order
+    assert (got.float() - out_a.float()).abs().max().item() <= 1e-2
+
+
+def test_strided_per_layer_cache_layout():
+    """A [B, N, S, D]-per-layer cache expressed through the strides of the 5-d view."""
+    w = wl.shrink(wl.get_config("c2"), S=500, L=2, steps=2)
+    data = wl.make_prefill(w, device="cpu")
+    perm = lambda t: t.permute(2, 0, 3, 1, 4).contiguous().permute(1, 3, 0, 2, 4)   # storage [L, B, N, S, D]
+    Kc, Vc, Qc = data["K"].cuda(), data["V"].cuda(), data["Q_obs"].cuda()
+    a, b = make_cache(w, 2), make_cache(w, 2)
+    K, V, Q = perm(Kc), perm(Vc), perm(Qc)
+    assert K.stride(1) == w.D
+    a.score_select(Q, K)
+    a.compact(K, V)
+    b.score_select(Qc, Kc)
+    b.compact(Kc, Vc)
+    st = wl.make_step(w, 0, device="cuda")
+    for c in (a, b):
+        c.append(st["k_new"], st["v_new"])
+    oa, ob = a.decode_attn(st["q"]), b.decode_attn(st["q"])
+    torch.cuda.synchronize()
+    assert torch.equal(a.idx_tensor(), b.idx_tensor())
+    assert torch.equal(a.k_thin, b.k_thin)
+    assert torch.equal(oa, ob)
+
+
+def test_state_machine_and_capacity():
+    from paper_2407_21018_b200 import binding as tk
+    w = wl.shrink(wl.get_config("c1"), S=128, steps=2)
+    data = wl.make_prefill(w, device="cuda")
+    c = make_cache(w, 2)
+    st = wl.make_step(w, 0, device="cuda")
+    with pytest.raises(tk.ThinKError) as e:
+        c.compact(data["K"], data["V"])
+    assert e.value.status == tk.ERR_STATE
+    with pytest.raises(tk.ThinKError) as e:
+        c.append(st["k_new"], st["v_new"])
+    assert e.value.status == tk.ERR_STATE
+    with pytest.raises(tk.ThinKError) as e:
+        c.decode_attn(st["q"])
+    assert e.value.status == tk.ERR_STATE
+    with pytest.raises(tk.ThinKError) as e:
+        c.score_select(data["Q_obs"], data["K"], layer0=1, nlayers=1)
+    assert e.value.status == tk.ERR_INVALID_ARG
+    c.score_select(data["Q_obs"], data["K"])
+    c.compact(data["K"], data["V"])
+    assert c.tail_len() == w.recent
+    c.append(st["k_new"], st["v_new"])
+    c.append(st["k_new"], st["v_new"])
+    with pytest.raises(tk.ThinKError) as e:
+        c.append(st["k_new"], st["v_new"])
+    assert e.value.status == tk.ERR_CAPACITY
+    assert c.tail_len() == w.recent + 2
+    torch.cuda.synchronize()
+    assert c.device_error() == 0
+
+
+def test_guard_bytes_untouched():
+    """Outputs stay inside their buffers: canaries after out / idx survive."""
+    w = wl.shrink(wl.get_config("c4"), S=300, L=1, B=3, steps=1)
+    data = wl.make_prefill(w, device="cuda")
+    c = make_cache(w, 1)
+    c.score_select(data["Q_obs"], data["K"])
+    c.compact(data["K"], data["V"])
+    st = wl.make_step(w, 0, device="cuda")
+    c.append(st["k_new"], st["v_new"])
+    n = st["q"].numel()
+    buf = torch.full((n + 64,), 7.0, dtype=st["q"].dtype, device="cuda")
+    c.decode_attn(st["q"], out=buf[:n].view_as(st["q"]))
+    torch.cuda.synchronize()
+    assert (buf[n:] == 7.0).all()
+    assert torch.isfinite(buf[:n].float()).all()
+
+
+def _sampled_full_size(name, units, steps_checked, lam=None):
+    """Full-size workload in the launch configuration the benchmark times; the oracle checks
+    sampled (b, layer, key head) units: literal + closed-form scores, selection, compacted keys and
+    the attention rows of the unit's query heads."""
+    w = wl.get_config(name)
+    if lam is not None:
+        w = dataclasses.replace(w, lam=lam)
+    data = wl.make_prefill(w, device="cuda")
+    K, V, Q = data["K"], data["V"], data["Q_obs"]
+    cache = make_cache(w, max(steps_checked) + 1)
+    cache.score_select(Q, K)
+    cache.compact(K, V)
+    torch.cuda.synchronize()
+    from paper_2407_21018_b200 import binding as tk
+    G = w.N_q // w.N_kv
+    idx_gpu = cache.idx_tensor().cpu().numpy().astype(np.int64)
+    sc_gpu = cache.scores_tensor().cpu().numpy()
+    heads = {}
+    for n, (b, l, h) in enumerate(units):
+        S_b = w.seq_lens[b]
+        Kh, Vh = to64(K[b, :S_b, l, h]), to64(V[b, :S_b, l, h])
+        Qg = np.stack([to64(Q[b, :, l, h * G + g]) for g in range(G)])
+        s = orc.score_closed_form(Qg, Kh)
+        if n == 0:
+            np.testing.assert_allclose(orc.score_literal(Qg, Kh), s, rtol=1e-12)
+        np.testing.assert_allclose(sc_gpu[b, l, h], s, rtol=1e-6)
+        idx = orc.select_top_T(s, cache.T)
+        if not (idx == idx_gpu[b, l, h]).all():
+            assert orc.near_tie(s, cache.T, 1e-6), f"idx mismatch at {(b, l, h)}"
+            idx = idx_gpu[b, l, h]
+        K_T, K_r = orc.compact_keys(Kh, idx, w.recent)
+        assert (to64(tk.k_thin_logical(cache, b, l, h)) == K_T).all()
+        heads[(b, l, h)] = dict(idx=idx, K_T=K_T, K_full=K_r, V=Vh)
+    worst = 0.0
+    for t in range(max(steps_checked) + 1):
+        st = wl.make_step(w, t, device="cuda")
+        cache.append(st["k_new"], st["v_new"])
+        out = cache.decode_attn(st["q"])
+        torch.cuda.synchronize()
+        for (b, l, h), d in heads.items():
+            d["K_full"] = np.vstack([d["K_full"], to64(st["k_new"][b, l, h])[None]])
+            d["V"] = np.vstack([d["V"], to64(st["v_new"][b, l, h])[None]])
+            if t in steps_checked:
+                for g in range(G):
+                    want = orc.decode_attention(to64(st["q"][b, l, h * G + g]), d["K_T"], d["idx"], d["K_full"], d["V"])
+                    worst = max(worst, assert_attn_close(to64(out[b, l, h * G + g]), want, w.dtype, f"{name} {(b, l, h, g)} t={t}"))
+        if t in steps_checked:
+            assert torch.isfinite(out.float()).all()
+    assert cache.device_error() == 0
+    return worst
+
+
+def test_c2_full_size_sampled():
+    _sampled_full_size("c2", [(0, 0, 0), (0, 13, 5), (0, 31, 7), (0, 7, 2)], {0, 1, 5})
+
+
+def test_c3_full_size_sampled():
+    _sampled_full_size("c3", [(0, 0, 0), (3, 31, 7), (1, 17, 3)], {0, 2})
+
+
+def test_c4_full_size_sampled():
+    _sampled_full_size("c4", [(0, 0, 0), (15, 31, 31), (7, 12, 19), (3, 5, 8)], {0, 3})
+
+
+def test_c5_full_size_sampled():
+    _sampled_full_size("c5", [(0, 0, 0), (0, 31, 7)], {0, 1})
