@@ -165,6 +165,33 @@ thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, 
 thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
                                void* stream);
 
+/* Score + select without any caller- or library-side allocation.  (The paper has no counterpart:
+ * this is a packaging variant of thinK_score_select, same kernel, same results.)
+ *
+ * Who needs it: code that may not call cudaMalloc where it runs -- a plugin inside a host
+ * application that hands out all device memory itself, a callback running under a memory pool that
+ * forbids side allocations, or a process whose memory budget was fixed at start-up.  Such a caller
+ * cannot provide the `workspace` that thinK_create asks for, so this call needs no handle and no
+ * workspace: its scratch (lengths, ticket counters, fp64 partial sums) is a fixed 8 MiB array
+ * compiled into the library.  Every GPU that loads the library holds those 8 MiB until exit.
+ *
+ *   cfg, seq_lens: as for thinK_cache_bytes (seq_lens on the HOST; copied with the stream).
+ *   q_obs, k, layer0, nlayers: as for thinK_score_select.
+ *   idx:    device out, uint8 [B, L, N_kv, T]; rows of the given layers are written.
+ *   scores: device out, fp64 [B, L, N_kv, D], or NULL.
+ *
+ * Limit: lengths + counters + 2 * B * nlayers * (N_kv*D) * 8 bytes per token split must fit in
+ * 8 MiB.  The call lowers its token split to fit; if even one split does not fit it launches nothing
+ * and returns THINK_ERR_CAPACITY -- pass fewer layers per call.
+ * The first call on a device looks up the array's device address (once per device; make that first
+ * call outside of any stream capture).  No cudaMalloc/cudaFree is called, here or later.
+ * All calls share the one array, which still holds the previous call's contents: the call rewrites
+ * the lengths and zeroes the tickets on `stream` before the kernel.  Two calls whose GPU work can
+ * overlap (different streams, or different host threads without ordering) race on it: order them. */
+thinK_status thinK_score_select_static(const thinK_config* cfg, const int32_t* seq_lens, thinK_tensor5 q_obs,
+                                       thinK_tensor5 k, int32_t layer0, int32_t nlayers, uint8_t* idx,
+                                       double* scores, void* stream);
+
 /* Tokens currently in the unpruned tail of `layer` (S_recent + appended), or -1. */
 int32_t thinK_tail_len(const thinK_cache* c, int32_t layer);
 

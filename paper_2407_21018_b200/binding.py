@@ -56,6 +56,8 @@ EXPORTS = {
     "thinK_compact": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_append": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_decode_attn": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_score_select_static": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32), Tensor5, Tensor5, C.c_int32,
+                                            C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
     "thinK_tail_len": (C.c_int32, [C.c_void_p, C.c_int32]),
     "thinK_device_error": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32)]),
     "thinK_destroy": (C.c_int, [C.c_void_p]),
@@ -113,6 +115,18 @@ def _stream_ptr(stream) -> int:
     if stream is None:
         stream = torch.cuda.current_stream()
     return stream.cuda_stream
+
+
+def score_select_static(cfg: Config, seq_lens: Sequence[int], q_obs: Optional[torch.Tensor], k: torch.Tensor,
+                        idx: torch.Tensor, scores: Optional[torch.Tensor] = None, layer0=0, nlayers=None, stream=None):
+    """thinK_score_select_static: same results as ThinKCache.score_select, but the library brings its
+    own fixed scratch, so nothing is allocated by the call (for callers that may not allocate device
+    memory).  `idx` (uint8) and `scores` (float64, optional) are caller-provided outputs."""
+    nlayers = cfg.L - layer0 if nlayers is None else nlayers
+    arr = (C.c_int32 * len(seq_lens))(*seq_lens)
+    _check(lib.thinK_score_select_static(C.byref(cfg), arr, tensor5(q_obs), tensor5(k), layer0, nlayers,
+                                         idx.data_ptr(), scores.data_ptr() if scores is not None else None,
+                                         _stream_ptr(stream)), "thinK_score_select_static")
 
 
 class ThinKCache:

@@ -6,6 +6,10 @@
 // 16-byte loads.  bf16 squares are exact in fp32; fp32 chains of 8 terms are flushed into fp64.
 // The CTA that arrives last for its (b, l, column block) -- an atomic ticket, nobody waits --
 // adds the partials in split order (deterministic), forms the scores and ranks each head.
+#include <string.h>
+
+#include <mutex>
+
 #include "think_internal.h"
 
 namespace think {
@@ -217,3 +221,111 @@ cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s) {
 }
 
 }  // namespace think
+
+// ---------------------------------------------------------------------------------------------
+// Score + select for callers that cannot allocate device memory.
+//
+// The kernel's scratch (per-sequence lengths, ticket counters, fp64 partial sums) lives in a fixed
+// array that is part of the library image: every GPU that loads the library holds these bytes until
+// the process exits.  Host code cannot use the array's name as an address -- it is only a host-side
+// handle of the symbol -- so the device address is looked up once per device with
+// cudaGetSymbolAddress and cached.
+// ---------------------------------------------------------------------------------------------
+#define THINK_STATIC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_think_static_scratch[THINK_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mu;
+void* g_scratch_addr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device (first use on a device resolves it).
+cudaError_t static_scratch(unsigned char** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_scratch_mu);
+  if (!g_scratch_addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_think_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (!p) return cudaErrorInvalidSymbol;
+    g_scratch_addr[dev] = p;
+  }
+  *out = (unsigned char*)g_scratch_addr[dev];
+  return cudaSuccess;
+}
+
+inline size_t up256(size_t x) { return (x + 255) & ~(size_t)255; }
+}  // namespace
+
+extern "C" thinK_status thinK_score_select_static(const thinK_config* cfg, const int32_t* seq_lens,
+                                                  thinK_tensor5 q_obs, thinK_tensor5 k, int32_t layer0,
+                                                  int32_t nlayers, uint8_t* idx, double* scores, void* stream) {
+  using namespace think;
+  if (!cfg || !seq_lens || !idx || !k.ptr) return THINK_ERR_INVALID_ARG;
+  if (cfg->B < 1 || cfg->L < 1 || cfg->N_kv < 1 || cfg->N_q < 1 || cfg->N_q % cfg->N_kv != 0 || cfg->S_obs < 1)
+    return THINK_ERR_INVALID_ARG;
+  if (cfg->dtype != THINK_BF16 && cfg->dtype != THINK_F32) return THINK_ERR_UNSUPPORTED;
+  if (cfg->D != 64 && cfg->D != 128) return THINK_ERR_UNSUPPORTED;
+  if (cfg->criterion < THINK_SCORE_QUERY_DRIVEN || cfg->criterion > THINK_SCORE_KEY_L1) return THINK_ERR_INVALID_ARG;
+  if (layer0 < 0 || nlayers < 1 || layer0 + nlayers > cfg->L || (int64_t)cfg->B * nlayers > 65535)
+    return THINK_ERR_INVALID_ARG;
+  if (cfg->criterion == THINK_SCORE_QUERY_DRIVEN && !q_obs.ptr) return THINK_ERR_INVALID_ARG;
+  const int T = thinK_T(cfg->lambda, cfg->D);
+  if (T < 1) return THINK_ERR_INVALID_ARG;
+  const int E = cfg->dtype == THINK_BF16 ? 2 : 4;
+  const thinK_tensor5* views[2] = {&k, &q_obs};
+  for (int v = 0; v < (cfg->criterion == THINK_SCORE_QUERY_DRIVEN ? 2 : 1); ++v) {
+    const int64_t st[4] = {views[v]->stride_b, views[v]->stride_s, views[v]->stride_l, views[v]->stride_n};
+    if (((uintptr_t)views[v]->ptr & 15) != 0) return THINK_ERR_INVALID_ARG;
+    for (int i = 0; i < 4; ++i)
+      if (st[i] < 0 || (st[i] * E) % 16 != 0) return THINK_ERR_INVALID_ARG;
+  }
+  int min_len = seq_lens[0];
+  for (int b = 0; b < cfg->B; ++b) {
+    if (seq_lens[b] < cfg->S_obs || seq_lens[b] > cfg->S_max) return THINK_ERR_INVALID_ARG;
+    min_len = seq_lens[b] < min_len ? seq_lens[b] : min_len;
+  }
+
+  ScoreParams p;
+  memset(&p, 0, sizeof(p));
+  const int CH = 16 / E;
+  p.NC = cfg->N_kv * cfg->D / CH;
+  p.CB = p.NC < kScoreThreads ? p.NC : kScoreThreads;
+  p.ncolblk = (p.NC + p.CB - 1) / p.CB;
+  p.RP = kScoreThreads / p.CB;
+  const int items = cfg->B * nlayers * p.ncolblk;
+  int nsplit = (kScoreTargetCtas + items - 1) / items;
+  int cap = min_len / (64 * p.RP);
+  if (cap < 1) cap = 1;
+  if (nsplit > cap) nsplit = cap;
+  // scratch: lengths | counters | partials; shrink the token split until it fits, else refuse
+  const size_t off_cnt = up256(sizeof(int32_t) * (size_t)cfg->B);
+  const size_t off_part = off_cnt + up256(sizeof(uint32_t) * (size_t)items);
+  const size_t per_split = (size_t)items * 2 * p.CB * CH * sizeof(double);
+  while (nsplit > 1 && off_part + per_split * nsplit > THINK_STATIC_SCRATCH_BYTES) --nsplit;
+  if (off_part + per_split * nsplit > THINK_STATIC_SCRATCH_BYTES) return THINK_ERR_CAPACITY;
+  p.nsplit = nsplit;
+
+  unsigned char* scratch = nullptr;
+  if (static_scratch(&scratch) != cudaSuccess) return THINK_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)stream;
+  // the array keeps whatever the previous call left: lengths are rewritten, tickets start at zero
+  if (cudaMemcpyAsync(scratch, seq_lens, sizeof(int32_t) * (size_t)cfg->B, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return THINK_ERR_CUDA;
+  if (cudaMemsetAsync(scratch + off_cnt, 0, sizeof(uint32_t) * (size_t)items, s) != cudaSuccess) return THINK_ERR_CUDA;
+
+  p.k = View5{k.ptr, k.stride_b, k.stride_s, k.stride_l, k.stride_n};
+  p.q = View5{q_obs.ptr, q_obs.stride_b, q_obs.stride_s, q_obs.stride_l, q_obs.stride_n};
+  p.seq_len = (const int32_t*)scratch;
+  p.counters = (uint32_t*)(scratch + off_cnt);
+  p.partials = (double*)(scratch + off_part);
+  p.idx = idx;
+  p.scores = scores;
+  p.B = cfg->B; p.L = cfg->L; p.N_kv = cfg->N_kv; p.G = cfg->N_q / cfg->N_kv; p.D = cfg->D; p.T = T;
+  p.S_obs = cfg->S_obs; p.layer0 = layer0; p.nlayers = nlayers; p.criterion = cfg->criterion;
+  if (launch_score(p, cfg->dtype, s) != cudaSuccess) return THINK_ERR_CUDA;
+  return THINK_OK;
+}
