@@ -152,7 +152,8 @@ def run_ours(args):
         E = lambda: torch.cuda.Event(enable_timing=True)
         return {"p0": E(), "p1": E(), "d0": [E() for _ in range(nsteps)], "d1": [E() for _ in range(nsteps)]}
 
-    for _ in range(max(3, args.warmup)):
+    n_warm = args.warmup if args.profile else max(3, args.warmup)
+    for _ in range(n_warm):
         one_pass()
     torch.cuda.synchronize()
 
@@ -253,7 +254,7 @@ def run_ours(args):
         line = {
             "metric": "ThinK hot path effective HBM GB/s (prefill score+select+compact, then decode append+attn; "
                       "algorithmic bytes / device time)",
-            "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": n_warm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": f"{w.name}: B={w.B} S={list(w.seq_lens) if len(set(w.seq_lens)) > 1 else w.seq_lens[0]} "
@@ -360,6 +361,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
+    ap.add_argument("--profile", action="store_true",
+                    help="for runs under ncu: take --warmup literally (fewer launches before the captured ones)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
