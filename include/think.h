@@ -105,15 +105,21 @@ const char* thinK_status_string(thinK_status s);
 /* Sizes of the buffers thinK_create needs.  `seq_lens` (host, [B]) are the
  * prompt lengths S_b; S_recent <= S_b, S_obs <= S_b <= S_max.
  *
- * Library layout of k_thin: for every (b, l, h) the S_p = S_b - S_recent prefix
- * tokens are cut into tiles of 64 tokens; a tile is stored channel-major,
- * [T][64] elements, rows of 64 tokens whose 16-byte chunks are XOR-swizzled with
- * (row & 7) so that one bulk copy lands it in shared memory bank-conflict free.
- * Logical element (token t, kept channel c) of head (b, l, h) sits at element
- *   ((thin_tile_base(b) + (l*N_kv + h)*n_tiles(b) + t/64) * T + c) * 64 + swz(c, t%64)
- * with n_tiles(b) = ceil(S_p(b)/64), thin_tile_base(b) = sum_{b'<b} L*N_kv*n_tiles(b'),
- * swz(c, u) = (((u*e/16) ^ (c & 7)) * 16 + (u*e)%16) / e,  e = bytes/element.
- * tail_k uses the same tile layout with all D channels: [B, L, N_kv, ceil(cap/64)][D][64],
+ * Library layout of k_thin and tail_k.  For every (b, l, h) the S_p = S_b - S_recent prefix tokens
+ * are cut into tiles of 64 tokens; tile t of head (b, l, h) is tile number
+ *   thin_tile_base(b) + (l*N_kv + h)*n_tiles(b) + t,   n_tiles(b) = ceil(S_p(b)/64),
+ *   thin_tile_base(b) = sum_{b'<b} L*N_kv*n_tiles(b'),
+ * and a tile holds Tp x 64 elements (tokens past S_p are zero).
+ *  - fp32: Tp = T; channel-major [T][64], rows of 64 tokens whose 16-byte chunks are XOR-swizzled with
+ *    (row & 7): element (token u, channel c) at c*64 + swz(c, u),
+ *    swz(c, u) = (((u*4/16) ^ (c & 7)) * 16 + (u*4)%16) / 4.
+ *  - bf16: Tp = T rounded up to a multiple of 8 (extra channels are zero); the tile is stored in the
+ *    operand order of the tensor-core instruction that consumes it: four 16-token steps of Tp*32
+ *    bytes; in a step, for each group s of 16 channels a 512-byte chunk with 16 bytes per lane i
+ *    (r = i/4, q = i%4): for jx = 0,1 the channel pairs (16s+2q, +1) and (16s+2q+8, +9) of token
+ *    16*step + 8*jx + r; a trailing group of 8 channels is a 256-byte block with 8 bytes per lane
+ *    (pair (16*n16+2q, +1) for jx = 0,1).
+ * tail_k uses the same tile layout with all D channels: [B, L, N_kv, ceil(cap/64)] tiles of D x 64,
  * cap = S_recent + max_new_tokens. */
 thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens, thinK_sizes* out);
 

@@ -216,25 +216,45 @@ class ThinKCache:
 
 
 # ---------------------------------------------------------------------------
-# Address arithmetic of the documented library layout (for readers of k_thin /
+# Address arithmetic of the documented library layouts (for readers of k_thin /
 # tail_k, e.g. tests): pure indexing, no arithmetic of the method.
 # ---------------------------------------------------------------------------
-def swz(c: int, u: int, e: int) -> int:
-    """Element offset of token u (0..63) in row c of a channel-major tile."""
-    byte = u * e
-    return ((((byte >> 4) ^ (c & 7)) << 4) | (byte & 15)) // e
+def padded_T(T: int, dtype_code: int) -> int:
+    """Rows stored per thin tile: bf16 pads T to a multiple of 8."""
+    return (T + 7) & ~7 if dtype_code == BF16 else T
 
 
-def unpack_tiles(raw: torch.Tensor, n_tiles: int, rows: int, n_tokens: int, dtype: torch.dtype) -> torch.Tensor:
-    """raw: flat tensor of `dtype` holding n_tiles tiles [rows][64] (swizzled);
-    returns the logical [n_tokens, rows] matrix."""
-    e = raw.element_size()
-    t = raw[: n_tiles * rows * TILE_TOKENS].view(n_tiles, rows, TILE_TOKENS)
-    c = torch.arange(rows, device=raw.device)[:, None]
-    u = torch.arange(TILE_TOKENS, device=raw.device)[None, :]
-    byte = u * e
-    off = ((((byte >> 4) ^ (c & 7)) << 4) | (byte & 15)) // e          # [rows, 64]
-    logical = torch.gather(t, 2, off[None].expand(n_tiles, -1, -1))    # [tile, row, u]
+def _offsets_f32(rows: int, device) -> torch.Tensor:
+    """Element offset of (row c, token u) in a channel-major swizzled fp32 tile [rows][64]."""
+    c = torch.arange(rows, device=device)[:, None]
+    u = torch.arange(TILE_TOKENS, device=device)[None, :]
+    byte = u * 4
+    return c * TILE_TOKENS + ((((byte >> 4) ^ (c & 7)) << 4) | (byte & 15)) // 4
+
+
+def _offsets_bf16(Cp: int, device) -> torch.Tensor:
+    """Element offset of (channel c, token u) in a bf16 tile of 64 tokens x Cp channels stored in
+    MMA-fragment order (see include/think.h)."""
+    c = torch.arange(Cp, device=device)[:, None]
+    u = torch.arange(TILE_TOKENS, device=device)[None, :]
+    n16 = Cp >> 4
+    step, jx, r = u >> 4, (u >> 3) & 1, u & 7
+    base = step * Cp * 32
+    s, w = c >> 4, c & 15
+    half, q, lo = w >> 3, (w & 7) >> 1, w & 1
+    main = base + s * 512 + (r * 4 + q) * 16 + (jx * 2 + half) * 4 + lo * 2
+    w8 = c - n16 * 16
+    q8, lo8 = w8 >> 1, w8 & 1
+    tail8 = base + n16 * 512 + (r * 4 + q8) * 8 + jx * 4 + lo8 * 2
+    return torch.where(c < n16 * 16, main, tail8) // 2
+
+
+def unpack_tiles(raw: torch.Tensor, n_tiles: int, rows: int, n_tokens: int) -> torch.Tensor:
+    """raw: flat tensor (bf16 or fp32) holding n_tiles key tiles of `rows` channels x 64 tokens in
+    the library layout of its dtype; returns the logical [n_tokens, rows] matrix."""
+    t = raw[: n_tiles * rows * TILE_TOKENS].view(n_tiles, rows * TILE_TOKENS)
+    off = _offsets_bf16(rows, raw.device) if raw.dtype == torch.bfloat16 else _offsets_f32(rows, raw.device)
+    logical = t[:, off.reshape(-1)].view(n_tiles, rows, TILE_TOKENS)           # [tile, channel, u]
     return logical.permute(0, 2, 1).reshape(n_tiles * TILE_TOKENS, rows)[:n_tokens]
 
 
@@ -245,8 +265,11 @@ def k_thin_logical(cache: ThinKCache, b: int, l: int, h: int) -> torch.Tensor:
     nt = [(s - c.S_recent + TILE_TOKENS - 1) // TILE_TOKENS for s in cache.seq_lens]
     base = sum(c.L * c.N_kv * x for x in nt[:b]) + (l * c.N_kv + h) * nt[b]
     flat = cache.k_thin.view(cache.torch_dtype)
-    per = cache.T * TILE_TOKENS
-    return unpack_tiles(flat[base * per:(base + nt[b]) * per], nt[b], cache.T, S_p, cache.torch_dtype)
+    Tp = padded_T(cache.T, c.dtype)
+    per = Tp * TILE_TOKENS
+    full = unpack_tiles(flat[base * per:(base + nt[b]) * per], nt[b], Tp, S_p)
+    assert Tp == cache.T or not full[:, cache.T:].any(), "padding rows of a thin tile must be zero"
+    return full[:, :cache.T]
 
 
 def tail_logical(cache: ThinKCache, b: int, l: int, h: int):
@@ -258,6 +281,6 @@ def tail_logical(cache: ThinKCache, b: int, l: int, h: int):
     unit = (b * c.L + l) * c.N_kv + h
     per = c.D * TILE_TOKENS
     flat = cache.tail_k.view(cache.torch_dtype)
-    keys = unpack_tiles(flat[unit * ttc * per:(unit + 1) * ttc * per], ttc, c.D, n, cache.torch_dtype)
+    keys = unpack_tiles(flat[unit * ttc * per:(unit + 1) * ttc * per], ttc, c.D, n)
     vals = cache.tail_v.view(cache.torch_dtype)[unit * cap * c.D:(unit * cap + n) * c.D].view(n, c.D)
     return keys, vals

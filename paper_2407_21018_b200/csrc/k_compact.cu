@@ -1,24 +1,25 @@
 // Key-cache compaction (paper Sec. 3.3): K_T[t][c] = K[t][idx[c]] for the pruned prefix, written
-// as channel-major 64-token tiles ([T][64], 16-byte chunks XOR-swizzled by row), plus the writer
-// of the unpruned tail (recent prompt rows at prefill, the new token at decode).
+// as 64-token tiles in the layout the decode kernels read (bf16: MMA-fragment order with T padded
+// to a multiple of 8 by zero rows; fp32: channel-major [T][64] with XOR-swizzled 16-byte chunks),
+// plus the writer of the unpruned tail (recent prompt rows at prefill, the new token at decode).
 #include "think_internal.h"
 
 namespace think {
 namespace {
 
 // One CTA builds one tile: 64 token rows of one head are staged in shared memory (padded pitch),
-// every thread then gathers 16 bytes' worth of tokens of one kept channel, and the finished tile
+// the threads gather the kept channels into the tile image in shared memory, and the finished
 // image leaves with coalesced 16-byte stores.
 template <typename Tin>
 __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
   constexpr int E = sizeof(Tin);
   constexpr int CH = 16 / E;             // elements per 16-byte chunk
   extern __shared__ __align__(16) unsigned char smem[];
-  const int D = p.D, T = p.T;
+  const int D = p.D, T = p.T, Tp = p.Tp;
   const int pitch = D * E + 16;          // bytes; odd number of 16-byte chunks per row
   unsigned char* s_in = smem;                                   // [64][pitch]
-  unsigned char* s_out = smem + kTileTokens * pitch;            // [T][64*E]
-  uint8_t* s_idx = (uint8_t*)(s_out + T * kTileTokens * E);     // [T]
+  unsigned char* s_out = smem + kTileTokens * pitch;            // tile image, Tp*64*E bytes
+  uint8_t* s_idx = (uint8_t*)(s_out + Tp * kTileTokens * E);    // [T]
 
   const int tile = blockIdx.x, h = blockIdx.y;
   const int b = blockIdx.z / p.nlayers, l = p.layer0 + blockIdx.z % p.nlayers;
@@ -42,21 +43,33 @@ __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
   }
   __syncthreads();
 
-  // item (j, c): tokens [j*CH, (j+1)*CH) of kept channel c; consecutive lanes take consecutive c
-  const int nj = kTileTokens / CH;
-  for (int item = tid; item < nj * T; item += blockDim.x) {
-    int j = item / T, c = item % T;
-    int ch = s_idx[c];
-    __align__(16) Tin tmp[CH];
+  if (E == 2) {
+    // item (u, cp): channel pair (2cp, 2cp+1) of token u -> one 32-bit word of the fragment image
+    const int npair = Tp / 2;
+    for (int item = tid; item < kTileTokens * npair; item += blockDim.x) {
+      const int u = item / npair, c = (item % npair) * 2;
+      uint32_t lo = 0, hi = 0;
+      if (c < T) lo = *(const uint16_t*)(s_in + u * pitch + s_idx[c] * 2);
+      if (c + 1 < T) hi = *(const uint16_t*)(s_in + u * pitch + s_idx[c + 1] * 2);
+      *(uint32_t*)(s_out + frag_elem_byte(Tp, c, u)) = lo | (hi << 16);
+    }
+  } else {
+    // item (j, c): tokens [j*CH, (j+1)*CH) of kept channel c; consecutive lanes take consecutive c
+    const int nj = kTileTokens / CH;
+    for (int item = tid; item < nj * T; item += blockDim.x) {
+      int j = item / T, c = item % T;
+      int ch = s_idx[c];
+      __align__(16) Tin tmp[CH];
 #pragma unroll
-    for (int i = 0; i < CH; ++i) tmp[i] = *(const Tin*)(s_in + (j * CH + i) * pitch + ch * E);
-    *(uint4*)(s_out + c * kTileTokens * E + ((j ^ (c & 7)) << 4)) = *(const uint4*)tmp;
+      for (int i = 0; i < CH; ++i) tmp[i] = *(const Tin*)(s_in + (j * CH + i) * pitch + ch * E);
+      *(uint4*)(s_out + c * kTileTokens * E + ((j ^ (c & 7)) << 4)) = *(const uint4*)tmp;
+    }
   }
   __syncthreads();
 
   const int64_t gtile = p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * ntiles + tile;
-  uint4* dst = (uint4*)((unsigned char*)p.k_thin + gtile * T * kTileTokens * E);
-  const int n16 = T * kTileTokens * E / 16;
+  uint4* dst = (uint4*)((unsigned char*)p.k_thin + gtile * Tp * kTileTokens * E);
+  const int n16 = Tp * kTileTokens * E / 16;
   for (int i = tid; i < n16; i += blockDim.x) dst[i] = ((const uint4*)s_out)[i];
 }
 
@@ -91,7 +104,8 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
 #pragma unroll
     for (int j = 0; j < CH; ++j) {
       int c = ck * CH + j;
-      *(Tin*)(tile + c * kTileTokens * E + tile_swz_bytes(c, uu, E)) = kk[j];
+      if (E == 2) *(Tin*)(tile + frag_elem_byte(p.D, c, uu)) = kk[j];
+      else *(Tin*)(tile + c * kTileTokens * E + tile_swz_bytes(c, uu, E)) = kk[j];
     }
   }
 }
@@ -102,7 +116,7 @@ cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cud
   if (max_tiles <= 0) return cudaSuccess;
   dim3 grid(max_tiles, p.N_kv, p.B * p.nlayers);
   const int E = dtype == THINK_BF16 ? 2 : 4;
-  size_t smem = (size_t)kTileTokens * (p.D * E + 16) + (size_t)p.T * kTileTokens * E + ((p.T + 15) & ~15);
+  size_t smem = (size_t)kTileTokens * (p.D * E + 16) + (size_t)p.Tp * kTileTokens * E + ((p.T + 15) & ~15);
   cudaError_t e;
   if (dtype == THINK_BF16) {
     e = cudaFuncSetAttribute(k_compact<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

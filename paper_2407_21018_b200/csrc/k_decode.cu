@@ -1,5 +1,6 @@
 // Decode attention over the two-part key cache (paper Sec. 3.3 / Fig. 2, attention of Sec. 3.2),
-// CUDA-core version for every dtype / head dimension / group size.
+// CUDA-core version.  It serves fp32 caches (logits in fp64); bf16 caches use the tensor-core kernel
+// in k_decode_mma.cu, whose key tiles are laid out differently.
 //
 // Work is the flat list of 64-token tiles of all (b, layer, key head) units: thin tiles [T][64]
 // of the pruned prefix first, then tail tiles [D][64] of the unpruned keys.  The grid is
@@ -83,7 +84,7 @@ __global__ void __launch_bounds__(kDecThreads) k_decode_generic(const DecodePara
   const long long f0 = (long long)cta * N / p.grid, f1 = (long long)(cta + 1) * N / p.grid;
   const int LH = p.nlayers * p.N_kv;
   const int ntt = p.n_tail_tiles;
-  const size_t rec_bytes = ((size_t)G * (8 + 4 + 4 * D) + 15) & ~(size_t)15;
+  const size_t rec_bytes = rec_size(D, G);
   const LT scale = (LT)(1.4426950408889634 / sqrt((double)D));
 
   long long f = f0;
@@ -240,7 +241,7 @@ __global__ void __launch_bounds__(kDecThreads) k_decode_generic(const DecodePara
       if (complete) {
         store_out(outp + g * D + d, O / Lsum);
       } else {
-        ((float*)(rec + G * 12))[g * D + d] = O;
+        ((float*)(rec + rec_o_off(G)))[g * D + d] = O;
         if (d == 0) { ((double*)rec)[g] = M; ((float*)(rec + G * 8))[g] = Lsum; }
       }
     }
@@ -269,7 +270,7 @@ __global__ void __launch_bounds__(kDecThreads) k_decode_generic(const DecodePara
             const uint8_t* r = p.records + ((size_t)ci * 2 + (cf0 >= ustart ? 0 : 1)) * rec_bytes;
             const float sc = ex2((float)(__ldcg((const double*)r + g) - M));
             Lsum += __ldcg((const float*)(r + G * 8) + g) * sc;
-            O += __ldcg((const float*)(r + G * 12) + g * D + d) * sc;
+            O += __ldcg((const float*)(r + rec_o_off(G)) + g * D + d) * sc;
           }
           store_out(outp + g * D + d, O / Lsum);
         }
@@ -293,28 +294,26 @@ int occ_one() {
   return n;
 }
 
-#define THINK_DISPATCH(FN, ...)                                                          \
-  do {                                                                                   \
-    if (dtype == THINK_BF16) {                                                           \
-      if (D == 128) { switch (G) { case 1: return FN<__nv_bfloat16, 128, 1>(__VA_ARGS__); \
-                                   case 2: return FN<__nv_bfloat16, 128, 2>(__VA_ARGS__); \
-                                   case 4: return FN<__nv_bfloat16, 128, 4>(__VA_ARGS__); \
-                                   case 8: return FN<__nv_bfloat16, 128, 8>(__VA_ARGS__); } } \
-      if (D == 64)  { switch (G) { case 1: return FN<__nv_bfloat16, 64, 1>(__VA_ARGS__);  \
-                                   case 2: return FN<__nv_bfloat16, 64, 2>(__VA_ARGS__);  \
-                                   case 4: return FN<__nv_bfloat16, 64, 4>(__VA_ARGS__);  \
-                                   case 8: return FN<__nv_bfloat16, 64, 8>(__VA_ARGS__); } } \
-    } else {                                                                             \
-      if (D == 128) { switch (G) { case 1: return FN<float, 128, 1>(__VA_ARGS__);         \
-                                   case 2: return FN<float, 128, 2>(__VA_ARGS__);         \
-                                   case 4: return FN<float, 128, 4>(__VA_ARGS__);         \
-                                   case 8: return FN<float, 128, 8>(__VA_ARGS__); } }     \
-      if (D == 64)  { switch (G) { case 1: return FN<float, 64, 1>(__VA_ARGS__);          \
-                                   case 2: return FN<float, 64, 2>(__VA_ARGS__);          \
-                                   case 4: return FN<float, 64, 4>(__VA_ARGS__);          \
-                                   case 8: return FN<float, 64, 8>(__VA_ARGS__); } }      \
-    }                                                                                    \
+#define THINK_DISPATCH(FN, ...)                                                      \
+  do {                                                                               \
+    if (D == 128) { switch (G) { case 1: return FN<float, 128, 1>(__VA_ARGS__);       \
+                                 case 2: return FN<float, 128, 2>(__VA_ARGS__);       \
+                                 case 4: return FN<float, 128, 4>(__VA_ARGS__);       \
+                                 case 8: return FN<float, 128, 8>(__VA_ARGS__); } }   \
+    if (D == 64)  { switch (G) { case 1: return FN<float, 64, 1>(__VA_ARGS__);        \
+                                 case 2: return FN<float, 64, 2>(__VA_ARGS__);        \
+                                 case 4: return FN<float, 64, 4>(__VA_ARGS__);        \
+                                 case 8: return FN<float, 64, 8>(__VA_ARGS__); } }    \
   } while (0)
+
+cudaError_t launch_f32(const DecodeParams& p, int D, int G, cudaStream_t s) {
+  THINK_DISPATCH(launch_one, p, s);
+  return cudaErrorInvalidValue;
+}
+int occ_f32(int D, int G) {
+  THINK_DISPATCH(occ_one);
+  return 0;
+}
 
 }  // namespace
 
@@ -323,16 +322,24 @@ bool decode_supported(int dtype, int D, int G) {
          (G == 1 || G == 2 || G == 4 || G == 8);
 }
 
+cudaError_t launch_decode_bf16(const DecodeParams& p, int D, int G, cudaStream_t s);
+cudaError_t decode_setup_bf16(int D, int G);
+int decode_warps_bf16();
+
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int D, int G, cudaStream_t s) {
-  THINK_DISPATCH(launch_one, p, s);
-  return cudaErrorInvalidValue;
+  return dtype == THINK_BF16 ? launch_decode_bf16(p, D, G, s) : launch_f32(p, D, G, s);
 }
 
-int decode_ctas_per_sm(int dtype, int D, int G) {
-  THINK_DISPATCH(occ_one);
-  return 0;
+cudaError_t decode_setup(int dtype, int D, int G) {
+  return dtype == THINK_BF16 ? decode_setup_bf16(D, G) : cudaSuccess;
 }
 
-size_t decode_record_bytes(int D, int G) { return ((size_t)G * (8 + 4 + 4 * D) + 15) & ~(size_t)15; }
+// CTAs of the decode kernel that fit on one SM (the bf16 kernel takes the whole shared memory).
+int decode_ctas_per_sm(int dtype, int D, int G) { return dtype == THINK_BF16 ? 1 : occ_f32(D, G); }
+
+// Workers per CTA: partial-state records are indexed by worker.
+int decode_workers_per_cta(int dtype) { return dtype == THINK_BF16 ? decode_warps_bf16() : 1; }
+
+size_t decode_record_bytes(int D, int G) { return rec_size(D, G); }
 
 }  // namespace think

@@ -21,7 +21,7 @@ struct Layout {            // byte offsets inside the workspace
 };
 
 struct Geometry {
-  int B, L, N_q, N_kv, D, G, T, S_obs, R, max_new, cap, tail_tiles_cap, E, dtype, criterion;
+  int B, L, N_q, N_kv, D, G, T, Tp, S_obs, R, max_new, cap, tail_tiles_cap, E, dtype, criterion;
   int NC, CB, ncolblk, RPmax;
   int64_t total_thin_tiles;    // over all (b, l, h)
   int max_thin_tiles;          // per (l, h) over b
@@ -42,7 +42,7 @@ thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geome
   if (T < 1) return THINK_ERR_INVALID_ARG;
   if ((int64_t)c->B * c->L > 65535) return THINK_ERR_UNSUPPORTED;
   g->B = c->B; g->L = c->L; g->N_q = c->N_q; g->N_kv = c->N_kv; g->D = c->D; g->G = c->N_q / c->N_kv;
-  g->T = T; g->S_obs = c->S_obs; g->R = c->S_recent; g->max_new = c->max_new_tokens; g->cap = c->S_recent + c->max_new_tokens;
+  g->T = T; g->Tp = padded_T(T, c->dtype); g->S_obs = c->S_obs; g->R = c->S_recent; g->max_new = c->max_new_tokens; g->cap = c->S_recent + c->max_new_tokens;
   if (g->cap < 1) g->cap = 1;
   g->tail_tiles_cap = (g->cap + kTileTokens - 1) / kTileTokens;
   g->dtype = c->dtype; g->E = c->dtype == THINK_BF16 ? 2 : 4; g->criterion = c->criterion;
@@ -139,7 +139,7 @@ thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens,
   Layout w;
   make_layout(g, &w);
   const size_t units = (size_t)g.B * g.L * g.N_kv;
-  out->k_thin = align_up((size_t)g.total_thin_tiles * g.T * kTileTokens * g.E, 256);
+  out->k_thin = align_up((size_t)g.total_thin_tiles * g.Tp * kTileTokens * g.E, 256);
   if (out->k_thin == 0) out->k_thin = 256;
   out->tail_k = align_up(units * g.tail_tiles_cap * (size_t)g.D * kTileTokens * g.E, 256);
   out->tail_v = align_up(units * g.cap * (size_t)g.D * g.E, 256);
@@ -184,10 +184,12 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
     return THINK_ERR_CUDA;
   }
   c->num_sms = prop.multiProcessorCount;
+  if (decode_setup(c->g.dtype, c->g.D, c->g.G) != cudaSuccess) { delete c; return THINK_ERR_CUDA; }
   int occ = decode_ctas_per_sm(c->g.dtype, c->g.D, c->g.G);
   if (occ < 1) { delete c; return THINK_ERR_CUDA; }
   c->decode_grid_max = c->num_sms * occ;
-  if (c->decode_grid_max > kMaxDecodeCtas) c->decode_grid_max = kMaxDecodeCtas;
+  const int wpc = decode_workers_per_cta(c->g.dtype);
+  if (c->decode_grid_max * wpc > kMaxDecodeCtas) c->decode_grid_max = kMaxDecodeCtas / wpc;
   // device tables
   const Geometry& g = c->g;
   bool ok = cudaMemset(c->ws, 0, c->w.header_bytes) == cudaSuccess;
@@ -254,7 +256,7 @@ thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int
   p.thin_tile_base = (const int64_t*)(c->ws + c->w.thin_tile_base);
   p.idx = (const uint8_t*)c->idx;
   p.k_thin = c->k_thin;
-  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.D = g.D; p.T = g.T; p.R = g.R;
+  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.D = g.D; p.T = g.T; p.Tp = g.Tp; p.R = g.R;
   p.layer0 = layer0; p.nlayers = nlayers;
   if (launch_compact(p, g.dtype, g.max_thin_tiles, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
   if (g.R > 0) {
@@ -323,7 +325,7 @@ thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t
   p.thin_tile_base = (const int64_t*)(c->ws + c->w.thin_tile_base);
   p.records = c->ws + c->w.decode_records;
   p.counters = (uint32_t*)(c->ws + c->w.decode_counters);
-  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.N_q = g.N_q; p.T = g.T; p.R = g.R; p.cap = g.cap;
+  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.N_q = g.N_q; p.T = g.T; p.Tp = g.Tp; p.R = g.R; p.cap = g.cap;
   p.tail_tiles_cap = g.tail_tiles_cap;
   p.n_tail = n_tail;
   p.n_tail_tiles = (n_tail + kTileTokens - 1) / kTileTokens;

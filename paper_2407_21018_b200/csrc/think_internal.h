@@ -41,7 +41,7 @@ struct CompactParams {
   const int64_t* thin_tile_base;
   const uint8_t* idx;
   void* k_thin;
-  int B, L, N_kv, D, T, R;
+  int B, L, N_kv, D, T, Tp, R;   // Tp = rows stored per thin tile (T padded to 8 for bf16)
   int layer0, nlayers;
 };
 
@@ -70,7 +70,7 @@ struct DecodeParams {
   const int64_t* thin_tile_base;
   uint8_t* records;
   uint32_t* counters;
-  int B, L, N_kv, N_q, T, R, cap, tail_tiles_cap;
+  int B, L, N_kv, N_q, T, Tp, R, cap, tail_tiles_cap;
   int n_tail;               // tokens in the tail
   int n_tail_tiles;
   int layer0, nlayers;
@@ -83,12 +83,41 @@ cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s);
 cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int D, int G, cudaStream_t s);
+cudaError_t decode_setup(int dtype, int D, int G);   // one-time per-process kernel attributes
+int decode_workers_per_cta(int dtype);
 bool decode_supported(int dtype, int D, int G);
 int decode_ctas_per_sm(int dtype, int D, int G);
 size_t decode_record_bytes(int D, int G);
 
+// Partial softmax state of one (worker, unit): double m[G] | float l[G] | pad to 16 | float o[G][D].
+constexpr __host__ __device__ int rec_o_off(int G) { return (G * 12 + 15) & ~15; }
+constexpr __host__ __device__ size_t rec_size(int D, int G) { return (size_t)rec_o_off(G) + (size_t)G * D * 4; }
+
+// Rows stored per thin tile: bf16 tiles are laid out in MMA-fragment order and pad T to a
+// multiple of 8 (zero rows); fp32 tiles are channel-major with exactly T rows.
+inline int padded_T(int T, int dtype) { return dtype == THINK_BF16 ? (T + 7) & ~7 : T; }
+
 // ---- device helpers ------------------------------------------------------
 #ifdef __CUDACC__
+// bf16 key tile of 64 tokens x Cp channels (Cp % 8 == 0) in MMA-fragment order.  The tile is four
+// 16-token steps of Cp*32 bytes.  Inside a step, for every 16-channel group s a 512-byte chunk holds,
+// per lane i (r = i/4, q = i%4), the B fragments of mma.m16n8k16 for the two 8-token halves jx:
+// [b0(jx=0) b1(jx=0) b0(jx=1) b1(jx=1)], b0 = channels 16s+2q,+1, b1 = channels 16s+2q+8,+9 of token
+// 16*step + 8*jx + r.  A trailing group of 8 channels (Cp % 16 == 8) is a 256-byte block with 8 bytes
+// per lane: [b(jx=0) b(jx=1)], channels 16*n16+2q,+1 (B fragments of mma.m16n8k8).
+// Returns the byte offset of element (token u, channel c).
+__host__ __device__ __forceinline__ int frag_elem_byte(int Cp, int c, int u) {
+  const int n16 = Cp >> 4;
+  const int step = u >> 4, jx = (u >> 3) & 1, r = u & 7;
+  const int base = step * Cp * 32;
+  if (c < n16 * 16) {
+    const int s = c >> 4, w = c & 15, half = w >> 3, q = (w & 7) >> 1, lo = w & 1;
+    return base + s * 512 + (r * 4 + q) * 16 + (jx * 2 + half) * 4 + lo * 2;
+  }
+  const int w = c - n16 * 16, q = w >> 1, lo = w & 1;
+  return base + n16 * 512 + (r * 4 + q) * 8 + jx * 4 + lo * 2;
+}
+
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 

@@ -49,7 +49,7 @@ def test_cache_bytes_and_memory_model(tk):
     s = tk.thinK_cache_bytes(cfg, [8192])
     T = 76
     n_tiles = math.ceil((8192 - 32) / 64)
-    assert s.k_thin == 32 * 8 * n_tiles * T * 64 * 2
+    assert s.k_thin == 32 * 8 * n_tiles * 80 * 64 * 2      # bf16 tiles pad T = 76 to 80 rows
     assert s.tail_k == 32 * 8 * math.ceil(96 / 64) * 128 * 64 * 2
     assert s.tail_v == 32 * 8 * 96 * 128 * 2
     assert s.idx == 32 * 8 * T
