@@ -43,13 +43,13 @@ __device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0
 
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
   // rows 8..15 of A (registers a1, a3) are zero: the group has at most 8 query heads
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ void mma1688(float (&d)[4], uint32_t a0, uint32_t b0) {
-  asm volatile(
+  asm(
       "mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a0), "r"(0u), "r"(b0));
@@ -67,14 +67,24 @@ __device__ __forceinline__ int worker_of(long long f, long long N, int nworkers)
   return (int)(((f + 1) * nworkers - 1) / N);
 }
 
-// One 16-token step in flight: where its keys and values come from.
-struct StepSrc {
-  const unsigned char* k;   // Cp*32 contiguous bytes
-  const unsigned char* v;   // first value row of the step
+// A run of consecutive 16-token steps of one kind (thin prefix tiles or unpruned tail tiles):
+// keys advance kstep bytes per step, values 16 rows per step.
+struct Region {
+  const unsigned char* k;   // keys of the first step (fragment order, kstep contiguous bytes per step)
+  const unsigned char* v;   // first value row
   long long vstride;        // bytes between value rows
-  int kbytes;               // Cp*32
-  int nrows;                // valid tokens in this step (1..16)
+  int kstep;                // Cp * 32
+  int ntok;                 // tokens in the region (the last step may be partial)
+  int n16;                  // 16-channel groups per key
+  bool has8;                // trailing 8-channel group
+  bool thin;
 };
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 
 template <int D, int G>
 __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParams p) {
@@ -98,6 +108,24 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
   const bool has8_thin = (Tp & 8) != 0;
   const size_t rec_bytes = rec_size(D, G);
   const float scale = 1.4426950408889634f / sqrtf((float)D);
+  // per-lane constants of the value path: which 16-byte chunk of which row this lane copies in
+  // iteration `it`, where it lands (XOR swizzle), and the ldmatrix row addresses per pair of n-tiles
+  constexpr int CPR = D * 2 / 16;          // 16-byte chunks per value row
+  constexpr int RPI = 32 / CPR;            // rows per copy iteration
+  constexpr int VIT = kStepTokens / RPI;   // copy iterations per step
+  const int vlane_row = lane / CPR, vlane_ck = lane % CPR;
+  int vdst_off[VIT];
+#pragma unroll
+  for (int it = 0; it < VIT; ++it) {
+    const int r = it * RPI + vlane_row;
+    vdst_off[it] = r * (D * 2) + ((vlane_ck ^ (r & 7)) << 4);
+  }
+  int vld_off[NT / 2];
+#pragma unroll
+  for (int np = 0; np < NT / 2; ++np) {
+    const int mi = lane >> 3, r = ((mi & 1) << 3) + (lane & 7), ck = 2 * np + (mi >> 1);
+    vld_off[np] = r * (D * 2) + ((ck ^ (r & 7)) << 4);
+  }
 
   long long f = f0;
   while (f < f1) {
@@ -128,42 +156,33 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
                                                          (int64_t)l * p.v.sl + (int64_t)h * p.v.sn);
     const unsigned char* vtail = (const unsigned char*)p.tail_v + unit_abs * p.cap * (int64_t)D * 2;
 
-    // tokens valid in tile j of this unit
-    auto tile_valid = [&](int j) {
-      return j < nthin ? min(kTileTokens, S_p - j * kTileTokens) : min(kTileTokens, p.n_tail - (j - nthin) * kTileTokens);
-    };
-    // source of step st of tile j
-    auto step_src = [&](int j, int st) {
-      StepSrc s;
-      const int nv = tile_valid(j) - st * kStepTokens;
-      s.nrows = nv < kStepTokens ? nv : kStepTokens;
-      if (j < nthin) {
-        s.kbytes = Tp * 32;
-        s.k = kthin + (int64_t)j * Tp * 128 + st * s.kbytes;
-        s.vstride = p.v.ss * 2;
-        s.v = vthin + (int64_t)(j * kTileTokens + st * kStepTokens) * s.vstride;
-      } else {
-        const int jt = j - nthin;
-        s.kbytes = D * 32;
-        s.k = ktail + (int64_t)jt * D * 128 + st * s.kbytes;
-        s.vstride = D * 2;
-        s.v = vtail + (int64_t)(jt * kTileTokens + st * kStepTokens) * s.vstride;
-      }
-      return s;
-    };
-    auto issue = [&](int slot, const StepSrc& s) {
-      const uint32_t kdst = ring + slot * kStage, vdst = kdst + kKSlot;
-      for (int i = lane; i * 16 < s.kbytes; i += 32) cp_async16(kdst + i * 16, s.k + i * 16, 16);
-      constexpr int CPR = D * 2 / 16;                  // 16-byte chunks per value row
-#pragma unroll
-      for (int it = 0; it < kStepTokens * CPR / 32; ++it) {
-        const int r = (it * 32 + lane) / CPR, ck = (it * 32 + lane) % CPR;
-        const bool ok = r < s.nrows;                   // rows past the valid tokens are zero-filled
-        cp_async16(vdst + r * (D * 2) + ((ck ^ (r & 7)) << 4), ok ? s.v + r * s.vstride + ck * 16 : s.v, ok ? 16 : 0);
-      }
-    };
+    // ---- the segment is at most two linear streams of 16-token steps: thin tiles, then tail tiles
+    Region r0{}, r1{};
+    int nreg = 0;
+    if (j0 < nthin) {
+      const int je = j1 < nthin ? j1 : nthin;
+      r0.kstep = Tp * 32;
+      r0.k = kthin + (int64_t)j0 * Tp * 128;
+      r0.vstride = p.v.ss * 2;
+      r0.v = vthin + (int64_t)j0 * kTileTokens * r0.vstride;
+      r0.ntok = min(S_p, je * kTileTokens) - j0 * kTileTokens;
+      r0.n16 = n16_thin; r0.has8 = has8_thin; r0.thin = true;
+      nreg = 1;
+    }
+    if (j1 > nthin) {
+      Region t;
+      const int jb = (j0 > nthin ? j0 : nthin) - nthin, je = j1 - nthin;
+      t.kstep = D * 32;
+      t.k = ktail + (int64_t)jb * D * 128;
+      t.vstride = D * 2;
+      t.v = vtail + (int64_t)jb * kTileTokens * t.vstride;
+      t.ntok = min(p.n_tail, je * kTileTokens) - jb * kTileTokens;
+      t.n16 = KS; t.has8 = false; t.thin = false;
+      if (nreg == 0) r0 = t; else r1 = t;
+      ++nreg;
+    }
 
-    // ---- query fragments (A operand).  qa[s] = channels 16s+2qd,+1 | qa[s+KS] = channels 16s+2qd+8,+9
+    // ---- query fragments (A operand): qa[s][0] = channels 16s+2qd,+1 ; qa[s][1] = channels 16s+2qd+8,+9
     const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q + ((int64_t)(b * p.nlayers + ll) * p.N_q + h * G) * D;
     const uint8_t* idx = p.idx + unit_abs * p.T;
     uint32_t qa[KS][2];
@@ -189,23 +208,41 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       }
       qa8 = (thin && has8_thin) ? q_pair(16 * n16_thin + 2 * qd, true) : 0u;
     };
-    bool q_is_thin = j0 < nthin;
-    load_q(q_is_thin);
 
-    // ---- online-softmax state of this worker for the unit (row = query head `row`)
+    // ---- online-softmax state of this worker for the unit (row = query head `row`), exp2 domain
     float m = -INFINITY, lsum = 0.f;
     float o[NT][4];
 #pragma unroll
     for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
 
-    // ---- software pipeline over the steps of tiles [j0, j1)
-    int ij = j0, ist = 0, islot = 0;                    // next step to issue
-    auto steps_of = [&](int j) { return (tile_valid(j) + kStepTokens - 1) / kStepTokens; };
-    int isteps = steps_of(j0);
+    // ---- producer side of the warp's ring: one step per call, pointers advance linearly
+    int ir = 0, itok = 0, islot = 0;
+    const unsigned char* ik = r0.k;
+    const unsigned char* iv = r0.v + vlane_row * r0.vstride + vlane_ck * 16;
     auto issue_next = [&]() {
-      if (ij < j1) {
-        issue(islot, step_src(ij, ist));
-        if (++ist == isteps) { ist = 0; ++ij; if (ij < j1) isteps = steps_of(ij); }
+      if (ir < nreg) {
+        const Region& R = ir ? r1 : r0;
+        const uint32_t kdst = ring + islot * kStage + lane * 16, vdst = ring + islot * kStage + kKSlot;
+        const int npiece = R.kstep >> 4;
+#pragma unroll
+        for (int n = 0; n < kKSlot / 512; ++n)
+          if (n * 32 + lane < npiece) cp_async16(kdst + n * 512, ik + lane * 16 + n * 512, 16);
+        const int nrows = R.ntok - itok;                // rows past the valid tokens are zero-filled
+        const unsigned char* vs = iv;
+#pragma unroll
+        for (int it = 0; it < VIT; ++it) {
+          const bool ok = it * RPI + vlane_row < nrows;
+          cp_async16(vdst + vdst_off[it], ok ? vs : R.v, ok ? 16 : 0);
+          vs += RPI * R.vstride;
+        }
+        itok += kStepTokens;
+        ik += R.kstep;
+        iv += kStepTokens * R.vstride;
+        if (itok >= R.ntok) {
+          ++ir; itok = 0;
+          ik = r1.k;
+          iv = r1.v + vlane_row * r1.vstride + vlane_ck * 16;
+        }
       }
       cp_commit();                                      // one group per call, possibly empty
       islot = islot + 1 == kStages ? 0 : islot + 1;
@@ -213,18 +250,17 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
 #pragma unroll
     for (int i = 0; i < kStages - 1; ++i) issue_next();
 
+    // ---- consumer side
     int cslot = 0;
-    for (int cj = j0; cj < j1; ++cj) {
-      const bool thin = cj < nthin;
-      if (thin != q_is_thin) { load_q(thin); q_is_thin = thin; }
-      const int nvalid = tile_valid(cj);
-      const int nsteps = (nvalid + kStepTokens - 1) / kStepTokens;
-      const int n16 = thin ? n16_thin : KS;
-      const bool has8 = thin && has8_thin;
-      for (int st = 0; st < nsteps; ++st) {
+    for (int cr = 0; cr < nreg; ++cr) {
+      const Region& R = cr ? r1 : r0;
+      load_q(R.thin);
+      const int n16 = R.n16;
+      const bool has8 = R.has8;
+      for (int ctok = 0; ctok < R.ntok; ctok += kStepTokens) {
         cp_wait<kStages - 2>();
         __syncwarp();
-        const uint32_t kbase = ring + cslot * kStage, vbase = kbase + kKSlot;
+        const uint32_t kbase = ring + cslot * kStage + lane * 16, vbase = ring + cslot * kStage + kKSlot;
         // S = q . K^T for the two 8-token halves of the step
         float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -232,43 +268,48 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
           if (s < n16) {
             uint4 kb;
             asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
-                         : "=r"(kb.x), "=r"(kb.y), "=r"(kb.z), "=r"(kb.w) : "r"(kbase + s * 512 + lane * 16));
+                         : "=r"(kb.x), "=r"(kb.y), "=r"(kb.z), "=r"(kb.w) : "r"(kbase + s * 512));
             mma16816(s0, qa[s][0], qa[s][1], kb.x, kb.y);
             mma16816(s1, qa[s][0], qa[s][1], kb.z, kb.w);
           }
         }
         if (has8) {
           uint2 kb;
-          asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(kb.x), "=r"(kb.y) : "r"(kbase + n16 * 512 + lane * 8));
+          asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];"
+                       : "=r"(kb.x), "=r"(kb.y) : "r"(kbase - lane * 8 + n16 * 512));
           mma1688(s0, qa8, kb.x);
           mma1688(s1, qa8, kb.y);
         }
-        // mask, scale into the exp2 domain, running max of this row over the quad
-        const int t0 = st * kStepTokens + 2 * qd;        // token (in tile) of s0[0]
-        float x00 = t0 < nvalid ? s0[0] * scale : -INFINITY;
-        float x01 = t0 + 1 < nvalid ? s0[1] * scale : -INFINITY;
-        float x10 = t0 + 8 < nvalid ? s1[0] * scale : -INFINITY;
-        float x11 = t0 + 9 < nvalid ? s1[1] * scale : -INFINITY;
-        float mx = fmaxf(fmaxf(x00, x01), fmaxf(x10, x11));
+        const int nrows = R.ntok - ctok;
+        if (nrows < kStepTokens) {                      // last step of the region: mask the missing tokens
+          const int t0 = 2 * qd;
+          if (t0 >= nrows) s0[0] = -INFINITY;
+          if (t0 + 1 >= nrows) s0[1] = -INFINITY;
+          if (t0 + 8 >= nrows) s1[0] = -INFINITY;
+          if (t0 + 9 >= nrows) s1[1] = -INFINITY;
+        }
+        // running max of this row over the quad, in the exp2 domain
+        float mx = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s1[0], s1[1]));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float mnew = fmaxf(m, mx);
-        const float sc = exp2f(m - mnew);
-        m = mnew;
-        const uint32_t pa0 = pack_bf16(exp2f(x00 - mnew), exp2f(x01 - mnew));
-        const uint32_t pa2 = pack_bf16(exp2f(x10 - mnew), exp2f(x11 - mnew));
-        // the denominator sums the rounded weights, so numerator and denominator agree
-        lsum = lsum * sc + (bf16lo(pa0) + bf16hi(pa0)) + (bf16lo(pa2) + bf16hi(pa2));
+        mx *= scale;
+        if (__any_sync(0xffffffffu, mx > m)) {          // some row's maximum grew: rescale the state
+          const float mnew = fmaxf(m, mx);
+          const float sc = ex2(m - mnew);
+          m = mnew;
+          lsum *= sc;
 #pragma unroll
-        for (int t = 0; t < NT; ++t) { o[t][0] *= sc; o[t][1] *= sc; }
+          for (int t = 0; t < NT; ++t) { o[t][0] *= sc; o[t][1] *= sc; }
+        }
+        const uint32_t pa0 = pack_bf16(ex2(fmaf(s0[0], scale, -m)), ex2(fmaf(s0[1], scale, -m)));
+        const uint32_t pa2 = pack_bf16(ex2(fmaf(s1[0], scale, -m)), ex2(fmaf(s1[1], scale, -m)));
+        // the denominator sums the rounded weights, so numerator and denominator agree
+        lsum += (bf16lo(pa0) + bf16hi(pa0)) + (bf16lo(pa2) + bf16hi(pa2));
         // O += P . V : value rows through ldmatrix.trans (tokens become the contraction index)
 #pragma unroll
         for (int np = 0; np < NT / 2; ++np) {
-          const int mi = lane >> 3;
-          const int r = ((mi & 1) << 3) + (lane & 7);
-          const int ck = 2 * np + (mi >> 1);
           uint32_t v0, v1, v2, v3;
-          ldmatrix_x4_trans(vbase + r * (D * 2) + ((ck ^ (r & 7)) << 4), v0, v1, v2, v3);
+          ldmatrix_x4_trans(vbase + vld_off[np], v0, v1, v2, v3);
           mma16816(o[2 * np], pa0, pa2, v0, v1);
           mma16816(o[2 * np + 1], pa0, pa2, v2, v3);
         }
