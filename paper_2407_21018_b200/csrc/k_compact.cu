@@ -43,17 +43,7 @@ __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
   }
   __syncthreads();
 
-  if (E == 2) {
-    // item (u, cp): channel pair (2cp, 2cp+1) of token u -> one 32-bit word of the fragment image
-    const int npair = Tp / 2;
-    for (int item = tid; item < kTileTokens * npair; item += blockDim.x) {
-      const int u = item / npair, c = (item % npair) * 2;
-      uint32_t lo = 0, hi = 0;
-      if (c < T) lo = *(const uint16_t*)(s_in + u * pitch + s_idx[c] * 2);
-      if (c + 1 < T) hi = *(const uint16_t*)(s_in + u * pitch + s_idx[c + 1] * 2);
-      *(uint32_t*)(s_out + frag_elem_byte(Tp, c, u)) = lo | (hi << 16);
-    }
-  } else {
+  {
     // item (j, c): tokens [j*CH, (j+1)*CH) of kept channel c; consecutive lanes take consecutive c
     const int nj = kTileTokens / CH;
     for (int item = tid; item < nj * T; item += blockDim.x) {
@@ -71,6 +61,70 @@ __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
   uint4* dst = (uint4*)((unsigned char*)p.k_thin + gtile * Tp * kTileTokens * E);
   const int n16 = Tp * kTileTokens * E / 16;
   for (int i = tid; i < n16; i += blockDim.x) dst[i] = ((const uint4*)s_out)[i];
+}
+
+// bf16 tiles in MMA-fragment order.  The 64 token rows are staged with cp.async (everything in
+// flight at once); then warp w builds the four 16-token steps w of the tile: for each group of 16
+// kept channels a lane gathers the eight elements of its 16-byte fragment piece (two tokens x four
+// channels) and the warp writes the 512-byte chunk straight to global memory.
+__global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int D = p.D, T = p.T, Tp = p.Tp;
+  const int pitch = D * 2 + 16;
+  unsigned char* s_in = smem;                                   // [64][pitch]
+  uint8_t* s_idx = smem + kTileTokens * pitch;                  // [Tp], padding channels -> 255
+  const int zb = gridDim.z - 1 - blockIdx.z;                    // last layers first: their keys are the
+  const int h = blockIdx.y;                                     // most recently scored, likely still in L2
+  const int b = zb / p.nlayers, l = p.layer0 + zb % p.nlayers;
+  const int S_p = p.seq_len[b] - p.R;
+  const int ntiles = (S_p + kTileTokens - 1) / kTileTokens;
+  if ((int)blockIdx.x >= ntiles) return;
+  const int tile = ntiles - 1 - blockIdx.x;
+  const int tok0 = tile * kTileTokens;
+  const int nvalid = min(kTileTokens, S_p - tok0);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+  for (int c = tid; c < Tp; c += 128) s_idx[c] = c < T ? p.idx[unit * T + c] : 255;
+  const __nv_bfloat16* src = (const __nv_bfloat16*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn;
+  const int cpr = D / 8;                 // 16-byte chunks per row
+  const uint32_t s_in_addr = (uint32_t)__cvta_generic_to_shared(s_in);
+  for (int i = tid; i < kTileTokens * cpr; i += 128) {
+    const int r = i / cpr, ck = i % cpr;
+    const bool ok = r < nvalid;          // rows past the prefix become zeros
+    const void* g = src + (int64_t)(tok0 + (ok ? r : 0)) * p.k.ss + ck * 8;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(s_in_addr + r * pitch + ck * 16), "l"(g), "r"(ok ? 16 : 0) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+
+  const int64_t gtile = p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * ntiles + tile;
+  unsigned char* dst = (unsigned char*)p.k_thin + gtile * Tp * 128 + warp * (Tp * 32);   // step = warp
+  const int r = lane >> 2, q = lane & 3;
+  const unsigned char* rowA = s_in + (warp * 16 + r) * pitch;
+  const unsigned char* rowB = rowA + 8 * pitch;
+  auto elem = [&](const unsigned char* row, int ch) -> uint32_t {
+    return ch == 255 ? 0u : (uint32_t)*(const uint16_t*)(row + ch * 2);
+  };
+  const int n16 = Tp >> 4;
+  for (int s = 0; s < n16; ++s) {
+    const int c0 = s_idx[16 * s + 2 * q], c1 = s_idx[16 * s + 2 * q + 1];
+    const int c8 = s_idx[16 * s + 2 * q + 8], c9 = s_idx[16 * s + 2 * q + 9];
+    uint4 v;
+    v.x = elem(rowA, c0) | (elem(rowA, c1) << 16);
+    v.y = elem(rowA, c8) | (elem(rowA, c9) << 16);
+    v.z = elem(rowB, c0) | (elem(rowB, c1) << 16);
+    v.w = elem(rowB, c8) | (elem(rowB, c9) << 16);
+    *(uint4*)(dst + s * 512 + lane * 16) = v;
+  }
+  if (Tp & 8) {
+    const int c0 = s_idx[16 * n16 + 2 * q], c1 = s_idx[16 * n16 + 2 * q + 1];
+    uint2 v;
+    v.x = elem(rowA, c0) | (elem(rowA, c1) << 16);
+    v.y = elem(rowB, c0) | (elem(rowB, c1) << 16);
+    *(uint2*)(dst + n16 * 512 + lane * 8) = v;
+  }
 }
 
 // Rows of unpruned keys and their values into the tail.  One thread moves one 16-byte chunk of
@@ -119,9 +173,8 @@ cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cud
   size_t smem = (size_t)kTileTokens * (p.D * E + 16) + (size_t)p.Tp * kTileTokens * E + ((p.T + 15) & ~15);
   cudaError_t e;
   if (dtype == THINK_BF16) {
-    e = cudaFuncSetAttribute(k_compact<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    k_compact<__nv_bfloat16><<<grid, 128, smem, s>>>(p);
+    smem = (size_t)kTileTokens * (p.D * 2 + 16) + ((p.Tp + 15) & ~15);
+    k_compact_bf16<<<grid, 128, smem, s>>>(p);
   } else {
     e = cudaFuncSetAttribute(k_compact<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;

@@ -24,8 +24,14 @@
 namespace think {
 namespace {
 
-constexpr int kWarps = 6;               // workers per CTA
-constexpr int kStages = 4;              // ring depth per warp (3 steps in flight)
+#ifndef THINK_DEC_WARPS
+#define THINK_DEC_WARPS 6
+#endif
+#ifndef THINK_DEC_STAGES
+#define THINK_DEC_STAGES 4
+#endif
+constexpr int kWarps = THINK_DEC_WARPS;  // workers per CTA
+constexpr int kStages = THINK_DEC_STAGES;  // ring depth per warp (kStages - 1 steps in flight)
 constexpr int kStepTokens = 16;
 constexpr int kKSlot = 4096;            // bytes: keys of one step at D = 128
 constexpr int kVSlot = 4096;            // bytes: 16 value rows at D = 128
@@ -34,7 +40,11 @@ constexpr int kSmemBytes = kWarps * kStages * kStage;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int src_bytes) {
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+// copies src_bytes (0 or 16) and zero-fills the rest of the 16 bytes
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, int src_bytes) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -216,31 +226,45 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
     for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
 
     // ---- producer side of the warp's ring: one step per call, pointers advance linearly
-    int ir = 0, itok = 0, islot = 0;
-    const unsigned char* ik = r0.k;
+    int ir = 0, islot = 0;
+    int i_left = r0.ntok;                               // tokens of the current region not yet issued
+    int i_kstep = r0.kstep;
+    long long i_vrow = r0.vstride;
+    const unsigned char* ikl = r0.k + lane * 16;
     const unsigned char* iv = r0.v + vlane_row * r0.vstride + vlane_ck * 16;
+    const unsigned char* i_vsafe = r0.v;
     auto issue_next = [&]() {
       if (ir < nreg) {
-        const Region& R = ir ? r1 : r0;
-        const uint32_t kdst = ring + islot * kStage + lane * 16, vdst = ring + islot * kStage + kKSlot;
-        const int npiece = R.kstep >> 4;
+        const uint32_t sb = ring + islot * kStage;
+        const uint32_t kd = sb + lane * 16;
+        const int nfull = i_kstep >> 9, krem = i_kstep & 511;       // 512-byte pieces of the key step
 #pragma unroll
-        for (int n = 0; n < kKSlot / 512; ++n)
-          if (n * 32 + lane < npiece) cp_async16(kdst + n * 512, ik + lane * 16 + n * 512, 16);
-        const int nrows = R.ntok - itok;                // rows past the valid tokens are zero-filled
+        for (int n = 0; n < D * 32 / 512; ++n)
+          if (n < nfull) cp_async16(kd + n * 512, ikl + n * 512);
+        if (lane * 16 < krem) cp_async16(kd + nfull * 512, ikl + nfull * 512);
         const unsigned char* vs = iv;
+        const long long rstep = RPI * i_vrow;
+        if (i_left >= kStepTokens) {
 #pragma unroll
-        for (int it = 0; it < VIT; ++it) {
-          const bool ok = it * RPI + vlane_row < nrows;
-          cp_async16(vdst + vdst_off[it], ok ? vs : R.v, ok ? 16 : 0);
-          vs += RPI * R.vstride;
+          for (int it = 0; it < VIT; ++it) {
+            cp_async16(sb + kKSlot + vdst_off[it], vs);
+            vs += rstep;
+          }
+        } else {                                        // last step of a region: zero-fill missing rows
+#pragma unroll
+          for (int it = 0; it < VIT; ++it) {
+            const bool ok = it * RPI + vlane_row < i_left;
+            cp_async16_zfill(sb + kKSlot + vdst_off[it], ok ? vs : i_vsafe, ok ? 16 : 0);
+            vs += rstep;
+          }
         }
-        itok += kStepTokens;
-        ik += R.kstep;
-        iv += kStepTokens * R.vstride;
-        if (itok >= R.ntok) {
-          ++ir; itok = 0;
-          ik = r1.k;
+        i_left -= kStepTokens;
+        ikl += i_kstep;
+        iv += kStepTokens * i_vrow;
+        if (i_left <= 0) {
+          ++ir;
+          i_left = r1.ntok; i_kstep = r1.kstep; i_vrow = r1.vstride; i_vsafe = r1.v;
+          ikl = r1.k + lane * 16;
           iv = r1.v + vlane_row * r1.vstride + vlane_ck * 16;
         }
       }
@@ -253,11 +277,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
     // ---- consumer side
     int cslot = 0;
     for (int cr = 0; cr < nreg; ++cr) {
-      const Region& R = cr ? r1 : r0;
-      load_q(R.thin);
-      const int n16 = R.n16;
-      const bool has8 = R.has8;
-      for (int ctok = 0; ctok < R.ntok; ctok += kStepTokens) {
+      const bool thin = cr ? r1.thin : r0.thin;
+      const int ntok = cr ? r1.ntok : r0.ntok;
+      load_q(thin);
+      const int n16 = thin ? n16_thin : KS;
+      const bool has8 = thin && has8_thin;
+      for (int left = ntok; left > 0; left -= kStepTokens) {
         cp_wait<kStages - 2>();
         __syncwarp();
         const uint32_t kbase = ring + cslot * kStage + lane * 16, vbase = ring + cslot * kStage + kKSlot;
@@ -280,13 +305,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
           mma1688(s0, qa8, kb.x);
           mma1688(s1, qa8, kb.y);
         }
-        const int nrows = R.ntok - ctok;
-        if (nrows < kStepTokens) {                      // last step of the region: mask the missing tokens
+        if (left < kStepTokens) {                       // last step of the region: mask the missing tokens
           const int t0 = 2 * qd;
-          if (t0 >= nrows) s0[0] = -INFINITY;
-          if (t0 + 1 >= nrows) s0[1] = -INFINITY;
-          if (t0 + 8 >= nrows) s1[0] = -INFINITY;
-          if (t0 + 9 >= nrows) s1[1] = -INFINITY;
+          if (t0 >= left) s0[0] = -INFINITY;
+          if (t0 + 1 >= left) s0[1] = -INFINITY;
+          if (t0 + 8 >= left) s1[0] = -INFINITY;
+          if (t0 + 9 >= left) s1[1] = -INFINITY;
         }
         // running max of this row over the quad, in the exp2 domain
         float mx = fmaxf(fmaxf(s0[0], s0[1]), fmaxf(s1[0], s1[1]));
@@ -348,24 +372,36 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       last = __shfl_sync(0xffffffffu, last, 0);
       if (last) {
         __threadfence();
-        for (int i = lane; i < G * D; i += 32) {
-          const int g = i / D, d = i % D;
-          float M = -INFINITY;
-          for (int ci = c_first; ci <= c_last; ++ci) {
-            const long long cf0 = (long long)ci * N / nworkers;
-            const uint8_t* r = p.records + ((size_t)ci * 2 + (cf0 >= ustart ? 0 : 1)) * rec_bytes;
-            M = fmaxf(M, (float)__ldcg((const double*)r + g));
+        // Merge in worker (= token) order.  Lane g < G owns the statistics of query head g; every
+        // lane owns G*D/32 output elements.  One round trip per contributor for the maxima, then one
+        // per contributor for its weights and all of this lane's output elements at once.
+        auto rec_of = [&](int ci) {
+          const long long cf0 = (long long)ci * N / nworkers;
+          return p.records + ((size_t)ci * 2 + (cf0 >= ustart ? 0 : 1)) * rec_bytes;
+        };
+        constexpr int EPL = G * D / 32;                  // elements per lane: i = lane + 32 k
+        float M = -INFINITY;
+        if (lane < G)
+          for (int ci = c_first; ci <= c_last; ++ci) M = fmaxf(M, (float)__ldcg((const double*)rec_of(ci) + lane));
+        float Lsum = 0.f, acc[EPL];
+#pragma unroll
+        for (int k = 0; k < EPL; ++k) acc[k] = 0.f;
+        for (int ci = c_first; ci <= c_last; ++ci) {
+          const uint8_t* r = rec_of(ci);
+          float ov[EPL];
+#pragma unroll
+          for (int k = 0; k < EPL; ++k) ov[k] = __ldcg((const float*)(r + rec_o_off(G)) + lane + 32 * k);
+          float w = 0.f;
+          if (lane < G) {
+            w = exp2f((float)__ldcg((const double*)r + lane) - M);
+            Lsum += __ldcg((const float*)(r + G * 8) + lane) * w;
           }
-          float Lsum = 0.f, O = 0.f;
-          for (int ci = c_first; ci <= c_last; ++ci) {
-            const long long cf0 = (long long)ci * N / nworkers;
-            const uint8_t* r = p.records + ((size_t)ci * 2 + (cf0 >= ustart ? 0 : 1)) * rec_bytes;
-            const float w = exp2f((float)__ldcg((const double*)r + g) - M);
-            Lsum += __ldcg((const float*)(r + G * 8) + g) * w;
-            O += __ldcg((const float*)(r + rec_o_off(G)) + g * D + d) * w;
-          }
-          outp[g * D + d] = __float2bfloat16_rn(O / Lsum);
+#pragma unroll
+          for (int k = 0; k < EPL; ++k) acc[k] = fmaf(ov[k], __shfl_sync(0xffffffffu, w, (lane + 32 * k) / D), acc[k]);
         }
+#pragma unroll
+        for (int k = 0; k < EPL; ++k)
+          outp[lane + 32 * k] = __float2bfloat16_rn(acc[k] / __shfl_sync(0xffffffffu, Lsum, (lane + 32 * k) / D));
         __syncwarp();
         if (lane == 0) p.counters[unit_call] = 0u;
       }

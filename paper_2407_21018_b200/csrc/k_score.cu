@@ -64,7 +64,7 @@ __device__ void select_head(const double* s, int D, int T, uint8_t* out, int lan
 }
 
 template <typename Tin, bool L1>
-__global__ void __launch_bounds__(kScoreThreads) k_colnorm_score_select(const ScoreParams p) {
+__global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const ScoreParams p) {
   constexpr int CH = Chunk<Tin>::CH;
   constexpr bool kBf16 = sizeof(Tin) == 2;
   __shared__ double red[kScoreThreads * CH];   // reused: row-lane reduction, then scores
@@ -83,9 +83,50 @@ __global__ void __launch_bounds__(kScoreThreads) k_colnorm_score_select(const Sc
   const int t0 = split * per;
   const int t1 = min(S_b, t0 + per);
 
-  double kacc[CH], qacc[CH];
+  // reduce one accumulator set over the row lanes of this CTA (fixed order) into this CTA's partial
+  const int CBE = p.CB * CH;  // elements per column block
+  double* my = p.partials + ((int64_t)(z * p.ncolblk + colblk) * p.nsplit + split) * 2 * CBE;
+  auto reduce_store = [&](const double (&acc)[CH], int pass) {
+    __syncthreads();
 #pragma unroll
-  for (int i = 0; i < CH; ++i) kacc[i] = 0.0, qacc[i] = 0.0;
+    for (int i = 0; i < CH; ++i) red[i * kScoreThreads + tid] = acc[i];   // tid = rl * CB + cl
+    __syncthreads();
+    if (rl == 0) {
+#pragma unroll
+      for (int i = 0; i < CH; ++i) {
+        double s = 0.0;
+        for (int r = 0; r < p.RP; ++r) s += red[i * kScoreThreads + r * p.CB + cl];
+        my[pass * CBE + cl * CH + i] = s;
+      }
+    }
+  };
+
+  {
+    // the window rows of the G query heads that share key head h (stacked)
+    double qacc[CH];
+#pragma unroll
+    for (int i = 0; i < CH; ++i) qacc[i] = 0.0;
+    if (active && p.criterion == THINK_SCORE_QUERY_DRIVEN) {
+      const Tin* qb = (const Tin*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl + j0;
+      const int nrows = p.S_obs * p.G;
+      for (int rr = split * p.RP + rl; rr < nrows; rr += p.nsplit * p.RP) {
+        int s = rr / p.G, g = rr % p.G;
+        uint4 v = ldg16(qb + (int64_t)s * p.q.ss + (int64_t)(h * p.G + g) * p.q.sn);
+        float x[CH];
+        Chunk<Tin>::unpack(v, x);
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          double d = (double)x[i];
+          qacc[i] = fma(d, d, qacc[i]);
+        }
+      }
+    }
+    reduce_store(qacc, 1);
+  }
+
+  double kacc[CH];
+#pragma unroll
+  for (int i = 0; i < CH; ++i) kacc[i] = 0.0;
 
   if (active) {
     const Tin* kb = (const Tin*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn + j0;
@@ -132,42 +173,8 @@ __global__ void __launch_bounds__(kScoreThreads) k_colnorm_score_select(const Sc
         kacc[i] = L1 ? kacc[i] + fabs(d) : fma(d, d, kacc[i]);
       }
     }
-    if (p.criterion == THINK_SCORE_QUERY_DRIVEN) {
-      // the window rows of the G query heads that share key head h (stacked)
-      const Tin* qb = (const Tin*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl + j0;
-      const int nrows = p.S_obs * p.G;
-      for (int rr = split * p.RP + rl; rr < nrows; rr += p.nsplit * p.RP) {
-        int s = rr / p.G, g = rr % p.G;
-        uint4 v = ldg16(qb + (int64_t)s * p.q.ss + (int64_t)(h * p.G + g) * p.q.sn);
-        float x[CH];
-        Chunk<Tin>::unpack(v, x);
-#pragma unroll
-        for (int i = 0; i < CH; ++i) {
-          double d = (double)x[i];
-          qacc[i] = fma(d, d, qacc[i]);
-        }
-      }
-    }
   }
-
-  // reduce over the row lanes of this CTA (fixed order), once for k and once for q
-  const int CBE = p.CB * CH;  // elements per column block
-  double* my = p.partials + ((int64_t)(z * p.ncolblk + colblk) * p.nsplit + split) * 2 * CBE;
-  for (int pass = 0; pass < 2; ++pass) {
-    double* acc = pass == 0 ? kacc : qacc;
-    __syncthreads();
-#pragma unroll
-    for (int i = 0; i < CH; ++i) red[tid * CH + i] = acc[i];   // tid = rl * CB + cl when rl < RP
-    __syncthreads();
-    if (rl == 0) {
-#pragma unroll
-      for (int i = 0; i < CH; ++i) {
-        double s = 0.0;
-        for (int r = 0; r < p.RP; ++r) s += red[(r * p.CB + cl) * CH + i];
-        my[pass * CBE + cl * CH + i] = s;
-      }
-    }
-  }
+  reduce_store(kacc, 0);
 
   // ticket: the last CTA of this (b, l, column block) finishes the job
   __threadfence();
@@ -180,11 +187,20 @@ __global__ void __launch_bounds__(kScoreThreads) k_colnorm_score_select(const Sc
 
   const double* base = p.partials + (int64_t)(z * p.ncolblk + colblk) * p.nsplit * 2 * CBE;
   const int ncols = min(CBE, (p.NC - colblk * p.CB) * CH);
+  __syncthreads();
   for (int c = tid; c < ncols; c += kScoreThreads) {
+    // partials are added in split order; loads are batched so their latencies overlap
     double kn = 0.0, qn = 0.0;
-    for (int s = 0; s < p.nsplit; ++s) {
-      kn += __ldcg(base + (int64_t)s * 2 * CBE + c);
-      qn += __ldcg(base + (int64_t)s * 2 * CBE + CBE + c);
+    for (int s0 = 0; s0 < p.nsplit; s0 += 8) {
+      double kv[8], qv[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const bool on = s0 + u < p.nsplit;
+        kv[u] = on ? __ldcg(base + (int64_t)(s0 + u) * 2 * CBE + c) : 0.0;
+        qv[u] = on ? __ldcg(base + (int64_t)(s0 + u) * 2 * CBE + CBE + c) : 0.0;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { kn += kv[u]; qn += qv[u]; }
     }
     double sc;
     if (p.criterion == THINK_SCORE_QUERY_DRIVEN) sc = sqrt(qn * kn);
