@@ -284,27 +284,36 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       const bool has8 = thin && has8_thin;
       for (int left = ntok; left > 0; left -= kStepTokens) {
         cp_wait<kStages - 2>();
-        __syncwarp();
+        __syncwarp();       // this step's data has landed; every lane is done with the previous slot
+        issue_next();       // refill that slot right away: the loads do not wait for this step's math
         const uint32_t kbase = ring + cslot * kStage + lane * 16, vbase = ring + cslot * kStage + kKSlot;
-        // S = q . K^T for the two 8-token halves of the step
+        // S = q . K^T for the two 8-token halves of the step; even and odd channel groups accumulate
+        // separately to halve the chain of dependent MMAs
         float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        float u0[4] = {0.f, 0.f, 0.f, 0.f}, u1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int s = 0; s < KS; ++s) {
           if (s < n16) {
             uint4 kb;
             asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                          : "=r"(kb.x), "=r"(kb.y), "=r"(kb.z), "=r"(kb.w) : "r"(kbase + s * 512));
-            mma16816(s0, qa[s][0], qa[s][1], kb.x, kb.y);
-            mma16816(s1, qa[s][0], qa[s][1], kb.z, kb.w);
+            if (s & 1) {
+              mma16816(u0, qa[s][0], qa[s][1], kb.x, kb.y);
+              mma16816(u1, qa[s][0], qa[s][1], kb.z, kb.w);
+            } else {
+              mma16816(s0, qa[s][0], qa[s][1], kb.x, kb.y);
+              mma16816(s1, qa[s][0], qa[s][1], kb.z, kb.w);
+            }
           }
         }
         if (has8) {
           uint2 kb;
           asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];"
                        : "=r"(kb.x), "=r"(kb.y) : "r"(kbase - lane * 8 + n16 * 512));
-          mma1688(s0, qa8, kb.x);
-          mma1688(s1, qa8, kb.y);
+          mma1688(u0, qa8, kb.x);
+          mma1688(u1, qa8, kb.y);
         }
+        s0[0] += u0[0]; s0[1] += u0[1]; s1[0] += u1[0]; s1[1] += u1[1];
         if (left < kStepTokens) {                       // last step of the region: mask the missing tokens
           const int t0 = 2 * qd;
           if (t0 >= left) s0[0] = -INFINITY;
@@ -337,8 +346,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
           mma16816(o[2 * np], pa0, pa2, v0, v1);
           mma16816(o[2 * np + 1], pa0, pa2, v2, v3);
         }
-        __syncwarp();                                   // every lane is done with the slot
-        issue_next();
         cslot = cslot + 1 == kStages ? 0 : cslot + 1;
       }
     }
