@@ -135,8 +135,11 @@ def run_ours(args):
     def one_pass(ev=None):
         if ev is not None:
             ev["p0"].record(stream)
-        cache.score_select(Q, K)
-        cache.compact(K, V)
+        if args.prefill == "fused":
+            cache.prefill(Q, K, V)
+        else:
+            cache.score_select(Q, K)
+            cache.compact(K, V)
         if ev is not None:
             ev["p1"].record(stream)
         for t in range(nsteps):
@@ -215,8 +218,11 @@ def run_ours(args):
             K.copy_(hK, non_blocking=True)
             V.copy_(hV, non_blocking=True)
             Q.copy_(hQ, non_blocking=True)
-            cache.score_select(Q, K)
-            cache.compact(K, V)
+            if args.prefill == "fused":
+                cache.prefill(Q, K, V)
+            else:
+                cache.score_select(Q, K)
+                cache.compact(K, V)
             for t in range(nsteps):
                 s = hs[t % nvar]
                 dq.copy_(s["q"], non_blocking=True)
@@ -259,7 +265,7 @@ def run_ours(args):
             "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": f"{w.name}: B={w.B} S={list(w.seq_lens) if len(set(w.seq_lens)) > 1 else w.seq_lens[0]} "
                                    f"L={w.L} heads={w.N_q}q/{w.N_kv}kv D={w.D} S_obs={w.S_obs} S_recent={w.recent} "
-                                   f"lambda={w.lam} T={T} decode_steps={nsteps}",
+                                   f"lambda={w.lam} T={T} decode_steps={nsteps} prefill={args.prefill}",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "l2": "inputs larger than L2 (K, V and the caches are each several L2 sizes)"},
             "decode": {"us_per_step": dec_mean_us, "GBps": dec_gbs, "frac_of_measured": dec_gbs / peak,
@@ -271,7 +277,7 @@ def run_ours(args):
                          "traffic": None},
             "clocks": clocks,
             "e2e": e2e,
-            "gpu_launches": args.steps * (2 + (1 if w.recent > 0 else 0) + 2 * nsteps),
+            "gpu_launches": args.steps * ((1 if args.prefill == "fused" else 2) + (1 if w.recent > 0 else 0) + 2 * nsteps),
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
@@ -358,6 +364,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--prefill", default="fused", choices=["fused", "split"],
+                    help="fused: thinK_prefill (one kernel); split: thinK_score_select + thinK_compact")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)

@@ -10,8 +10,8 @@
  * ("Observation Window"); the most recent S_recent prompt tokens and all newly
  * decoded tokens keep all D key channels (Sec. 3.3).
  *
- * Call order:   thinK_cache_bytes -> thinK_create -> thinK_score_select ->
- *               thinK_compact -> { thinK_append -> thinK_decode_attn }* -> thinK_destroy
+ * Call order:   thinK_cache_bytes -> thinK_create -> thinK_score_select -> thinK_compact
+ *               (or thinK_prefill for both) -> { thinK_append -> thinK_decode_attn }* -> thinK_destroy
  *
  * Conventions that hold for every entry point
  *  - All tensor pointers are DEVICE pointers unless marked "host".  The caller
@@ -152,6 +152,17 @@ thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tenso
  * thinK_decode_attn reads them in place on every step. */
 thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0, int32_t nlayers,
                            void* stream);
+
+/* Prefill in one call: thinK_score_select followed by thinK_compact for the same layers, with the
+ * same results (scores may differ in the last bits: the partial sums are grouped differently).
+ * For bf16 caches the two steps run as ONE persistent kernel that reads each head's keys from HBM
+ * once: a head is scored by a team of thread blocks and compacted one head later, while its keys
+ * are still in L2.  fp32 caches, and caches where some sequence has no pruned prefix, run the two
+ * steps back to back.  The fused kernel waits (bounded) on per-head flags; should a wait expire,
+ * the device error word is set (see thinK_device_error) and the cache contents are undefined.
+ * Arguments as for thinK_score_select / thinK_compact. */
+thinK_status thinK_prefill(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0,
+                           int32_t nlayers, void* stream);
 
 /* Decode, Sec. 3.3: the new token's key and value join the unpruned tail.
  * k_new, v_new: dense [B, nlayers, N_kv, D].  Every layer of the cache must be

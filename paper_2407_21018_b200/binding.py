@@ -54,6 +54,7 @@ EXPORTS = {
     "thinK_create": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32)] + [C.c_void_p] * 6 + [C.POINTER(C.c_void_p)]),
     "thinK_score_select": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_compact": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_prefill": (C.c_int, [C.c_void_p, Tensor5, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_append": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_decode_attn": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_score_select_static": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32), Tensor5, Tensor5, C.c_int32,
@@ -168,6 +169,14 @@ class ThinKCache:
         self._v = v   # borrowed by the library: keep it alive
         _check(lib.thinK_compact(self.handle, tensor5(k), tensor5(v), layer0, nlayers, _stream_ptr(stream)),
                "thinK_compact")
+
+    def prefill(self, q_obs: Optional[torch.Tensor], k: torch.Tensor, v: torch.Tensor, layer0=0, nlayers=None,
+                stream=None):
+        """score_select + compact in one call (one fused kernel for bf16 caches)."""
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        self._v = v   # borrowed by the library: keep it alive
+        _check(lib.thinK_prefill(self.handle, tensor5(q_obs), tensor5(k), tensor5(v), layer0, nlayers,
+                                 _stream_ptr(stream)), "thinK_prefill")
 
     def append(self, k_new: torch.Tensor, v_new: torch.Tensor, layer0=0, nlayers=None, stream=None):
         nlayers = self.cfg.L - layer0 if nlayers is None else nlayers

@@ -223,6 +223,20 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
 
 }  // namespace
 
+// CTAs of the score kernel that are resident per SM (the grid is sized to one wave)
+int score_ctas_per_sm(int dtype, int criterion) {
+  int n = 0;
+  cudaError_t e;
+  const bool l1 = criterion == THINK_SCORE_KEY_L1;
+  if (dtype == THINK_BF16)
+    e = l1 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_colnorm_score_select<__nv_bfloat16, true>, kScoreThreads, 0)
+           : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_colnorm_score_select<__nv_bfloat16, false>, kScoreThreads, 0);
+  else
+    e = l1 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_colnorm_score_select<float, true>, kScoreThreads, 0)
+           : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_colnorm_score_select<float, false>, kScoreThreads, 0);
+  return e == cudaSuccess ? n : 0;
+}
+
 cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s) {
   dim3 grid(p.nsplit, p.ncolblk, p.B * p.nlayers);
   const bool l1 = p.criterion == THINK_SCORE_KEY_L1;

@@ -96,15 +96,20 @@ def compare_cache(cache, o: orc.ThinKOracle, units=None, where=""):
         assert (to64(vf) == o.V_all[b][l][h][S_p:]).all(), f"{where} tail values differ at {(b, l, h)}"
 
 
-def run_case(w: wl.Workload, steps=None, criterion=0, check_cache=True):
-    """Whole path on both sides.  Returns dict of statistics."""
+def run_case(w: wl.Workload, steps=None, criterion=0, check_cache=True, fused=False):
+    """Whole path on both sides.  Returns dict of statistics.  `fused`: prefill through
+    thinK_prefill (one call) instead of thinK_score_select + thinK_compact."""
     steps = w.steps if steps is None else steps
     data = wl.make_prefill(w, device="cpu")
     K, V, Q = data["K"].cuda(), data["V"].cuda(), data["Q_obs"].cuda()
     cache = make_cache(w, steps, criterion)
-    cache.score_select(Q if criterion == 0 else None, K)
-    cache.compact(K, V)
+    if fused:
+        cache.prefill(Q if criterion == 0 else None, K, V)
+    else:
+        cache.score_select(Q if criterion == 0 else None, K)
+        cache.compact(K, V)
     torch.cuda.synchronize()
+    assert cache.device_error() == 0
 
     o = make_oracle(w)
     K64, V64, Q64 = to64(data["K"]), to64(data["V"]), to64(data["Q_obs"])

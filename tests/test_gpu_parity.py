@@ -32,6 +32,48 @@ def test_shrunk_configs(name, S, L, B, steps):
     run_case(w)
 
 
+@pytest.mark.parametrize("name,S,L,B,steps", [
+    ("c2", 2048 + 37, 3, 1, 2),
+    ("c3", 1500, 2, 2, 2),
+    ("c4", 700, 2, 5, 2),            # ragged, T = 51 (trailing group of 8 channels)
+    ("c5", 9000, 1, 1, 2),
+    ("c1", 300, 1, 1, 2),            # fp32: thinK_prefill runs the two kernels back to back
+])
+def test_fused_prefill(name, S, L, B, steps):
+    """thinK_prefill (single persistent kernel for bf16) against the oracle."""
+    w = wl.shrink(wl.get_config(name), S=S, L=L, B=B, steps=steps)
+    run_case(w, fused=True)
+
+
+@pytest.mark.parametrize("R,criterion", [(0, 0), (1, 0), (32, 1), (32, 2)])
+def test_fused_prefill_variants(R, criterion):
+    w = dataclasses.replace(wl.shrink(wl.get_config("c2"), S=1100, L=2, steps=2), S_recent=R)
+    run_case(w, fused=True, criterion=criterion)
+
+
+def test_fused_prefill_equals_two_pass_and_repeats():
+    """Same idx and the same key-cache bytes as score_select + compact; a second fused call on the
+    same handle (new epoch, re-used tickets and flags) gives the same bytes again."""
+    w = wl.shrink(wl.get_config("c4"), S=1300, L=2, B=3, steps=1)
+    data = wl.make_prefill(w, device="cuda")
+    a, b = make_cache(w, 1), make_cache(w, 1)
+    a.score_select(data["Q_obs"], data["K"])
+    a.compact(data["K"], data["V"])
+    for _ in range(2):
+        b.k_thin.zero_()
+        b.prefill(data["Q_obs"], data["K"], data["V"])
+        torch.cuda.synchronize()
+        assert b.device_error() == 0
+        assert torch.equal(a.idx_tensor(), b.idx_tensor())
+        assert torch.equal(a.k_thin, b.k_thin)
+    # per-layer fused calls
+    c = make_cache(w, 1)
+    for l in (1, 0):
+        c.prefill(data["Q_obs"], data["K"], data["V"], layer0=l, nlayers=1)
+    torch.cuda.synchronize()
+    assert torch.equal(a.idx_tensor(), c.idx_tensor()) and torch.equal(a.k_thin, c.k_thin)
+
+
 @pytest.mark.parametrize("lam", [0.0, 0.25, 0.75])
 def test_lambda_sweep(lam):
     w = wl.shrink(wl.get_config("c5"), S=1000, L=1, steps=3, lam=lam)
@@ -211,9 +253,9 @@ def _sampled_full_size(name, units, steps_checked, lam=None):
     data = wl.make_prefill(w, device="cuda")
     K, V, Q = data["K"], data["V"], data["Q_obs"]
     cache = make_cache(w, max(steps_checked) + 1)
-    cache.score_select(Q, K)
-    cache.compact(K, V)
+    cache.prefill(Q, K, V)           # the launch configuration the benchmark times
     torch.cuda.synchronize()
+    assert cache.device_error() == 0
     from paper_2407_21018_b200 import binding as tk
     G = w.N_q // w.N_kv
     idx_gpu = cache.idx_tensor().cpu().numpy().astype(np.int64)
