@@ -364,7 +364,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--decode-steps", type=int, default=None)
-    ap.add_argument("--prefill", default="fused", choices=["fused", "split"],
+    ap.add_argument("--prefill", default="split", choices=["fused", "split"],
                     help="fused: thinK_prefill (one kernel); split: thinK_score_select + thinK_compact")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
