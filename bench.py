@@ -29,6 +29,9 @@ sys.path.insert(0, ROOT)
 from paper_2407_21018_b200 import workloads as wl  # noqa: E402
 
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes (read + write) of ONE launch of the decode kernel from an ncu capture of the current
+# kernel (profiles/k_decode_mma_c2_ncu.md); configs without a capture report null.
+NCU_DECODE_TRAFFIC_BYTES = {"c2": 880.0e6}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -272,9 +275,9 @@ def run_ours(args):
                        "frac_of_nominal_8TBps": dec_gbs / NOMINAL_HBM_GBS, "bytes_per_step": dec_bytes_mean},
             "prefill": {"us": pre_us, "GBps": pre_gbs, "frac_of_measured": pre_gbs / peak,
                         "frac_of_nominal_8TBps": pre_gbs / NOMINAL_HBM_GBS, "bytes": pre_b},
-            "roofline": {"kernel": "k_decode_attn", "bound": "hbm", "achieved": dec_gbs, "peak": peak,
+            "roofline": {"kernel": "k_decode_mma" if w.dtype == "bf16" else "k_decode_generic", "bound": "hbm", "achieved": dec_gbs, "peak": peak,
                          "peak_source": f"of {peak_src}", "unit": "GB/s", "frac": dec_gbs / peak,
-                         "traffic": None},
+                         "traffic": NCU_DECODE_TRAFFIC_BYTES.get(w.name), "traffic_unit": "bytes per launch"},
             "clocks": clocks,
             "e2e": e2e,
             "gpu_launches": args.steps * ((1 if args.prefill == "fused" else 2) + (1 if w.recent > 0 else 0) + 2 * nsteps),
