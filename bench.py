@@ -32,6 +32,8 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) of ONE launch of the decode kernel from an ncu capture of the current
 # kernel (profiles/k_decode_mma_c2_ncu.md); configs without a capture report null.
 NCU_DECODE_TRAFFIC_BYTES = {"c2": 880.0e6}
+# DRAM bytes of the prefill kernels of one pass (score + compact; profiles/k_*_c2_ncu.md): K crosses HBM twice.
+NCU_PREFILL_TRAFFIC_BYTES = {"c2": 1379.9e6}
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -138,11 +140,8 @@ def run_ours(args):
     def one_pass(ev=None):
         if ev is not None:
             ev["p0"].record(stream)
-        if args.prefill == "fused":
-            cache.prefill(Q, K, V)
-        else:
-            cache.score_select(Q, K)
-            cache.compact(K, V)
+        cache.score_select(Q, K)
+        cache.compact(K, V)
         if ev is not None:
             ev["p1"].record(stream)
         for t in range(nsteps):
@@ -221,11 +220,8 @@ def run_ours(args):
             K.copy_(hK, non_blocking=True)
             V.copy_(hV, non_blocking=True)
             Q.copy_(hQ, non_blocking=True)
-            if args.prefill == "fused":
-                cache.prefill(Q, K, V)
-            else:
-                cache.score_select(Q, K)
-                cache.compact(K, V)
+            cache.score_select(Q, K)
+            cache.compact(K, V)
             for t in range(nsteps):
                 s = hs[t % nvar]
                 dq.copy_(s["q"], non_blocking=True)
@@ -268,19 +264,22 @@ def run_ours(args):
             "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": f"{w.name}: B={w.B} S={list(w.seq_lens) if len(set(w.seq_lens)) > 1 else w.seq_lens[0]} "
                                    f"L={w.L} heads={w.N_q}q/{w.N_kv}kv D={w.D} S_obs={w.S_obs} S_recent={w.recent} "
-                                   f"lambda={w.lam} T={T} decode_steps={nsteps} prefill={args.prefill}",
+                                   f"lambda={w.lam} T={T} decode_steps={nsteps}",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "l2": "inputs larger than L2 (K, V and the caches are each several L2 sizes)"},
             "decode": {"us_per_step": dec_mean_us, "GBps": dec_gbs, "frac_of_measured": dec_gbs / peak,
                        "frac_of_nominal_8TBps": dec_gbs / NOMINAL_HBM_GBS, "bytes_per_step": dec_bytes_mean},
             "prefill": {"us": pre_us, "GBps": pre_gbs, "frac_of_measured": pre_gbs / peak,
-                        "frac_of_nominal_8TBps": pre_gbs / NOMINAL_HBM_GBS, "bytes": pre_b},
+                        "frac_of_nominal_8TBps": pre_gbs / NOMINAL_HBM_GBS, "bytes": pre_b,
+                        "dram_bytes_ncu": NCU_PREFILL_TRAFFIC_BYTES.get(w.name),
+                        "dram_GBps": (NCU_PREFILL_TRAFFIC_BYTES[w.name] / (pre_us * 1e-6) / 1e9
+                                      if w.name in NCU_PREFILL_TRAFFIC_BYTES else None)},
             "roofline": {"kernel": "k_decode_mma" if w.dtype == "bf16" else "k_decode_generic", "bound": "hbm", "achieved": dec_gbs, "peak": peak,
                          "peak_source": f"of {peak_src}", "unit": "GB/s", "frac": dec_gbs / peak,
                          "traffic": NCU_DECODE_TRAFFIC_BYTES.get(w.name), "traffic_unit": "bytes per launch"},
             "clocks": clocks,
             "e2e": e2e,
-            "gpu_launches": args.steps * ((1 if args.prefill == "fused" else 2) + (1 if w.recent > 0 else 0) + 2 * nsteps),
+            "gpu_launches": args.steps * (2 + (1 if w.recent > 0 else 0) + 2 * nsteps),
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
@@ -367,8 +366,6 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--decode-steps", type=int, default=None)
-    ap.add_argument("--prefill", default="split", choices=["fused", "split"],
-                    help="fused: thinK_prefill (one kernel); split: thinK_score_select + thinK_compact")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)

@@ -153,14 +153,8 @@ thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tenso
 thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0, int32_t nlayers,
                            void* stream);
 
-/* Prefill in one call: thinK_score_select followed by thinK_compact for the same layers, with the
- * same results (scores may differ in the last bits: the partial sums are grouped differently).
- * For bf16 caches the two steps run as ONE persistent kernel that reads each head's keys from HBM
- * once: a head is scored by a team of thread blocks and compacted one head later, while its keys
- * are still in L2.  fp32 caches, and caches where some sequence has no pruned prefix, run the two
- * steps back to back.  The fused kernel waits (bounded) on per-head flags; should a wait expire,
- * the device error word is set (see thinK_device_error) and the cache contents are undefined.
- * Arguments as for thinK_score_select / thinK_compact. */
+/* Prefill in one call: thinK_score_select followed by thinK_compact for the same layers on the
+ * same stream (Sec. 3.2 + 3.3).  Arguments as for those two calls. */
 thinK_status thinK_prefill(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0,
                            int32_t nlayers, void* stream);
 

@@ -172,7 +172,7 @@ class ThinKCache:
 
     def prefill(self, q_obs: Optional[torch.Tensor], k: torch.Tensor, v: torch.Tensor, layer0=0, nlayers=None,
                 stream=None):
-        """score_select + compact in one call (one fused kernel for bf16 caches)."""
+        """score_select + compact in one call."""
         nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
         self._v = v   # borrowed by the library: keep it alive
         _check(lib.thinK_prefill(self.handle, tensor5(q_obs), tensor5(k), tensor5(v), layer0, nlayers,

@@ -16,7 +16,6 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // byte offsets inside the workspace
   size_t seq_len, cum_thin, thin_tile_base, error, score_counters, decode_counters;
-  size_t pf_tickets, pf_flags, pf_partials, pf_gpartials;
   size_t score_partials, decode_records, total;
   size_t header_bytes;     // everything before score_partials (initialised by thinK_create)
 };
@@ -76,14 +75,7 @@ void make_layout(const Geometry& g, Layout* w) {
   w->error = o;            o = align_up(o + 256, 256);
   w->score_counters = o;   o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.ncolblk, 256);
   w->decode_counters = o;  o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.N_kv, 256);
-  // fused prefill: tickets per head slab (one per reduction group + one), flags per head slab
-  const size_t units = (size_t)g.B * g.L * g.N_kv;
-  const size_t max_groups = (size_t)(kSMs * 2 + 15) / 16 + 1;
-  w->pf_tickets = o;       o = align_up(o + sizeof(uint32_t) * units * (max_groups + 1), 256);
-  w->pf_flags = o;         o = align_up(o + sizeof(uint32_t) * units, 256);
   w->header_bytes = o;
-  w->pf_partials = o;      o = align_up(o + sizeof(double) * (size_t)kSMs * 2 * 2 * 2 * g.D, 256);
-  w->pf_gpartials = o;     o = align_up(o + sizeof(double) * (size_t)kSMs * 2 * 2 * 2 * g.D, 256);
   w->score_partials = o;
   // a call splits tokens so that items * nsplit <= target + items
   const size_t slots = (size_t)kScoreTargetCtas + (size_t)g.B * g.L * g.ncolblk;
@@ -118,8 +110,6 @@ struct thinK_cache {
   bool have_v;
   int num_sms, decode_grid_max;
   int score_capacity;                       // resident CTAs of the score kernel on this device
-  int prefill_ctas_per_sm;                  // 0: fused prefill unavailable (fp32, or it does not fit)
-  uint32_t prefill_epoch;
 };
 
 extern "C" {
@@ -203,8 +193,6 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
   if (c->decode_grid_max * wpc > kMaxDecodeCtas) c->decode_grid_max = kMaxDecodeCtas / wpc;
   c->score_capacity = c->num_sms * score_ctas_per_sm(c->g.dtype, c->g.criterion);
   if (c->score_capacity < 1) { delete c; return THINK_ERR_CUDA; }
-  c->prefill_ctas_per_sm = c->g.dtype == THINK_BF16 ? prefill_max_ctas_per_sm(c->g.D, c->g.Tp) : 0;
-  c->prefill_epoch = 0;
   // device tables
   const Geometry& g = c->g;
   bool ok = cudaMemset(c->ws, 0, c->w.header_bytes) == cudaSuccess;
@@ -303,59 +291,9 @@ static thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, 
 
 thinK_status thinK_prefill(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0,
                            int32_t nlayers, void* stream) {
-  if (!c) return THINK_ERR_INVALID_ARG;
-  if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
-  const Geometry& g = c->g;
-  if (!check_view(k, g.E) || !check_view(v, g.E)) return THINK_ERR_INVALID_ARG;
-  if (g.criterion == THINK_SCORE_QUERY_DRIVEN && !check_view(q_obs, g.E)) return THINK_ERR_INVALID_ARG;
-  if (c->have_v && memcmp(&c->v, &v, sizeof(v)) != 0) return THINK_ERR_INVALID_ARG;
-  int min_len = g.seq_len[0], max_len = g.seq_len[0];
-  for (int b = 1; b < g.B; ++b) {
-    min_len = g.seq_len[b] < min_len ? g.seq_len[b] : min_len;
-    max_len = g.seq_len[b] > max_len ? g.seq_len[b] : max_len;
-  }
-  // the fused kernel needs a pruned prefix in every sequence; otherwise (and for fp32) run the two passes
-  if (c->prefill_ctas_per_sm < 1 || min_len - g.R < 1) {
-    thinK_status st = thinK_score_select(c, q_obs, k, layer0, nlayers, stream);
-    if (st != THINK_OK) return st;
-    return thinK_compact(c, k, v, layer0, nlayers, stream);
-  }
-  PrefillParams p;
-  memset(&p, 0, sizeof(p));
-  p.k = to_view(k); p.q = to_view(q_obs);
-  p.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
-  p.thin_tile_base = (const int64_t*)(c->ws + c->w.thin_tile_base);
-  p.idx = (uint8_t*)c->idx; p.scores = (double*)c->scores; p.k_thin = c->k_thin;
-  p.partials = (double*)(c->ws + c->w.pf_partials);
-  p.gpartials = (double*)(c->ws + c->w.pf_gpartials);
-  p.tickets = (uint32_t*)(c->ws + c->w.pf_tickets);
-  p.flags = (uint32_t*)(c->ws + c->w.pf_flags);
-  p.error = (uint32_t*)(c->ws + c->w.error);
-  p.epoch = ++c->prefill_epoch;
-  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.G = g.G; p.D = g.D; p.T = g.T; p.Tp = g.Tp; p.S_obs = g.S_obs; p.R = g.R;
-  p.layer0 = layer0; p.nlayers = nlayers; p.criterion = g.criterion;
-  p.nslabs = g.B * nlayers * g.N_kv;
-  // teams: ~448 tokens per member, two slabs per team resident in L2 (64 MB of it), every CTA used
-  int grid_max = c->num_sms * c->prefill_ctas_per_sm;
-  if (grid_max > kSMs * 2) grid_max = kSMs * 2;
-  const double slab_bytes = (double)max_len * g.D * g.E;
-  int nt_l2 = (int)(64.0 * 1024 * 1024 / (2.0 * slab_bytes));
-  if (nt_l2 < 1) nt_l2 = 1;
-  int ts = (max_len + 447) / 448;
-  if (ts < 1) ts = 1;
-  if (ts > grid_max) ts = grid_max;
-  int nt = grid_max / ts;
-  if (nt > nt_l2) nt = nt_l2;
-  if (nt > p.nslabs) nt = p.nslabs;
-  if (nt < 1) nt = 1;
-  ts = grid_max / nt;
-  const int ts_cap = (min_len - g.R + kTileTokens - 1) / kTileTokens;   // at least one prefix tile per member
-  if (ts > ts_cap) ts = ts_cap;
-  if (ts < 1) ts = 1;
-  p.TS = ts; p.NT = nt;
-  if (launch_prefill_fused(p, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
-  for (int l = layer0; l < layer0 + nlayers; ++l) c->scored[l] = 1;
-  return seed_tail(c, k, v, layer0, nlayers, stream);
+  thinK_status st = thinK_score_select(c, q_obs, k, layer0, nlayers, stream);
+  if (st != THINK_OK) return st;
+  return thinK_compact(c, k, v, layer0, nlayers, stream);
 }
 
 thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, int32_t layer0, int32_t nlayers,

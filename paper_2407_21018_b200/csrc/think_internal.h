@@ -45,24 +45,6 @@ struct CompactParams {
   int layer0, nlayers;
 };
 
-struct PrefillParams {       // fused score + select + compact (bf16)
-  View5 k, q;
-  const int32_t* seq_len;
-  const int64_t* thin_tile_base;
-  uint8_t* idx;
-  double* scores;
-  void* k_thin;
-  double* partials;         // [NT][2][TS][2][D]
-  double* gpartials;        // [NT][2][ngroups][2][D]
-  uint32_t* tickets;        // [slabs][ngroups + 1], zero between calls
-  uint32_t* flags;          // [slabs], compared with epoch
-  uint32_t* error;
-  uint32_t epoch;
-  int B, L, N_kv, G, D, T, Tp, S_obs, R;
-  int layer0, nlayers, criterion;
-  int TS, NT, nslabs;       // team size, teams, head slabs of this call
-};
-
 struct TailWriteParams {
   View5 k, v;               // sources
   int src_layer_base;       // layer index subtracted before applying sl
@@ -101,10 +83,6 @@ cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s);
 int score_ctas_per_sm(int dtype, int criterion);
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s);
 cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s);
-cudaError_t launch_prefill_fused(const PrefillParams& p, cudaStream_t s);
-size_t prefill_smem_bytes(int D, int Tp);
-int prefill_max_ctas_per_sm(int D, int Tp);
-int prefill_group_size();
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int D, int G, cudaStream_t s);
 cudaError_t decode_setup(int dtype, int D, int G);   // one-time per-process kernel attributes
 int decode_workers_per_cta(int dtype);

@@ -37,10 +37,10 @@ def test_shrunk_configs(name, S, L, B, steps):
     ("c3", 1500, 2, 2, 2),
     ("c4", 700, 2, 5, 2),            # ragged, T = 51 (trailing group of 8 channels)
     ("c5", 9000, 1, 1, 2),
-    ("c1", 300, 1, 1, 2),            # fp32: thinK_prefill runs the two kernels back to back
+    ("c1", 300, 1, 1, 2),            # fp32
 ])
 def test_fused_prefill(name, S, L, B, steps):
-    """thinK_prefill (single persistent kernel for bf16) against the oracle."""
+    """thinK_prefill (score_select + compact in one call) against the oracle."""
     w = wl.shrink(wl.get_config(name), S=S, L=L, B=B, steps=steps)
     run_case(w, fused=True)
 
@@ -52,8 +52,8 @@ def test_fused_prefill_variants(R, criterion):
 
 
 def test_fused_prefill_equals_two_pass_and_repeats():
-    """Same idx and the same key-cache bytes as score_select + compact; a second fused call on the
-    same handle (new epoch, re-used tickets and flags) gives the same bytes again."""
+    """Same idx and the same key-cache bytes as score_select + compact; a second call on the same
+    handle gives the same bytes again."""
     w = wl.shrink(wl.get_config("c4"), S=1300, L=2, B=3, steps=1)
     data = wl.make_prefill(w, device="cuda")
     a, b = make_cache(w, 1), make_cache(w, 1)
@@ -66,7 +66,7 @@ def test_fused_prefill_equals_two_pass_and_repeats():
         assert b.device_error() == 0
         assert torch.equal(a.idx_tensor(), b.idx_tensor())
         assert torch.equal(a.k_thin, b.k_thin)
-    # per-layer fused calls
+    # per-layer calls
     c = make_cache(w, 1)
     for l in (1, 0):
         c.prefill(data["Q_obs"], data["K"], data["V"], layer0=l, nlayers=1)
