@@ -137,6 +137,97 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
     vld_off[np] = r * (D * 2) + ((ck ^ (r & 7)) << 4);
   }
 
+  // ---- producer side of the warp's ring.  It walks the worker's whole tile range [f0, f1) on its own,
+  // region after region (thin tiles of a unit, then its tail tiles, then the next unit), so the ring stays
+  // full across unit boundaries; the consumer below follows the same sequence.
+  long long pf = f0;                                  // first tile not yet handed to the producer
+  int islot = 0, i_left = 0, i_kstep = 0;
+  long long i_vrow = 0;
+  const unsigned char* ikl = nullptr;
+  const unsigned char* iv = nullptr;
+  const unsigned char* i_vsafe = nullptr;
+  auto p_next_region = [&]() {                        // load the region that starts at tile pf (pf < f1)
+    int lo = 0, hi = p.B - 1;
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      long long cm = (long long)LH * (p.cum_thin[mid] + (long long)mid * ntt);
+      if (cm <= pf) lo = mid; else hi = mid - 1;
+    }
+    const int b = lo;
+    const int nthin = p.cum_thin[b + 1] - p.cum_thin[b];
+    const int tpu = nthin + ntt;
+    const long long rem = pf - (long long)LH * (p.cum_thin[b] + (long long)b * ntt);
+    const int u_in_b = (int)(rem / tpu), j0 = (int)(rem % tpu);
+    const int l = p.layer0 + u_in_b / p.N_kv, h = u_in_b % p.N_kv;
+    const long long uend = pf - j0 + tpu;
+    const int j1 = j0 + (int)((f1 < uend ? f1 : uend) - pf);
+    const int64_t unit_abs = ((int64_t)b * p.L + l) * p.N_kv + h;
+    const unsigned char *k0, *v0;
+    int ntiles;
+    if (j0 < nthin) {
+      const int je = j1 < nthin ? j1 : nthin;
+      ntiles = je - j0;
+      i_kstep = Tp * 32;
+      i_vrow = p.v.ss * 2;
+      k0 = (const unsigned char*)p.k_thin + (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * nthin + j0) * (int64_t)Tp * 128;
+      v0 = (const unsigned char*)((const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn) +
+           (int64_t)j0 * kTileTokens * i_vrow;
+      i_left = min(p.seq_len[b] - p.R, je * kTileTokens) - j0 * kTileTokens;
+    } else {
+      const int jb = j0 - nthin, je = j1 - nthin;
+      ntiles = je - jb;
+      i_kstep = D * 32;
+      i_vrow = D * 2;
+      k0 = (const unsigned char*)p.tail_k + (unit_abs * p.tail_tiles_cap + jb) * (int64_t)D * 128;
+      v0 = (const unsigned char*)p.tail_v + (unit_abs * p.cap + (int64_t)jb * kTileTokens) * D * 2;
+      i_left = min(p.n_tail, je * kTileTokens) - jb * kTileTokens;
+    }
+    ikl = k0 + lane * 16;
+    iv = v0 + vlane_row * i_vrow + vlane_ck * 16;
+    i_vsafe = v0;
+    pf += ntiles;
+  };
+  p_next_region();
+  auto issue_next = [&]() {
+    if (i_left > 0) {
+      const uint32_t sb = ring + islot * kStage;
+      const uint32_t kd = sb + lane * 16;
+      const int nfull = i_kstep >> 9, krem = i_kstep & 511;       // 512-byte pieces of the key step
+#pragma unroll
+      for (int n = 0; n < D * 32 / 512; ++n)
+        if (n < nfull) cp_async16(kd + n * 512, ikl + n * 512);
+      if (lane * 16 < krem) cp_async16(kd + nfull * 512, ikl + nfull * 512);
+      const unsigned char* vs = iv;
+      const long long rstep = RPI * i_vrow;
+      if (i_left >= kStepTokens) {
+#pragma unroll
+        for (int it = 0; it < VIT; ++it) {
+          cp_async16(sb + kKSlot + vdst_off[it], vs);
+          vs += rstep;
+        }
+      } else {                                        // last step of a region: zero-fill missing rows
+#pragma unroll
+        for (int it = 0; it < VIT; ++it) {
+          const bool ok = it * RPI + vlane_row < i_left;
+          cp_async16_zfill(sb + kKSlot + vdst_off[it], ok ? vs : i_vsafe, ok ? 16 : 0);
+          vs += rstep;
+        }
+      }
+      i_left -= kStepTokens;
+      ikl += i_kstep;
+      iv += kStepTokens * i_vrow;
+      if (i_left <= 0) {
+        i_left = 0;
+        if (pf < f1) p_next_region();
+      }
+    }
+    cp_commit();                                      // one group per call, possibly empty
+    islot = islot + 1 == kStages ? 0 : islot + 1;
+  };
+#pragma unroll 1
+  for (int i = 0; i < kStages - 1; ++i) issue_next();
+  int cslot = 0;                                      // consumer's slot, in step with the producer's
+
   long long f = f0;
   while (f < f1) {
     // ---- unit that owns tile f
@@ -225,57 +316,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
 #pragma unroll
     for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
 
-    // ---- producer side of the warp's ring: one step per call, pointers advance linearly
-    int ir = 0, islot = 0;
-    int i_left = r0.ntok;                               // tokens of the current region not yet issued
-    int i_kstep = r0.kstep;
-    long long i_vrow = r0.vstride;
-    const unsigned char* ikl = r0.k + lane * 16;
-    const unsigned char* iv = r0.v + vlane_row * r0.vstride + vlane_ck * 16;
-    const unsigned char* i_vsafe = r0.v;
-    auto issue_next = [&]() {
-      if (ir < nreg) {
-        const uint32_t sb = ring + islot * kStage;
-        const uint32_t kd = sb + lane * 16;
-        const int nfull = i_kstep >> 9, krem = i_kstep & 511;       // 512-byte pieces of the key step
-#pragma unroll
-        for (int n = 0; n < D * 32 / 512; ++n)
-          if (n < nfull) cp_async16(kd + n * 512, ikl + n * 512);
-        if (lane * 16 < krem) cp_async16(kd + nfull * 512, ikl + nfull * 512);
-        const unsigned char* vs = iv;
-        const long long rstep = RPI * i_vrow;
-        if (i_left >= kStepTokens) {
-#pragma unroll
-          for (int it = 0; it < VIT; ++it) {
-            cp_async16(sb + kKSlot + vdst_off[it], vs);
-            vs += rstep;
-          }
-        } else {                                        // last step of a region: zero-fill missing rows
-#pragma unroll
-          for (int it = 0; it < VIT; ++it) {
-            const bool ok = it * RPI + vlane_row < i_left;
-            cp_async16_zfill(sb + kKSlot + vdst_off[it], ok ? vs : i_vsafe, ok ? 16 : 0);
-            vs += rstep;
-          }
-        }
-        i_left -= kStepTokens;
-        ikl += i_kstep;
-        iv += kStepTokens * i_vrow;
-        if (i_left <= 0) {
-          ++ir;
-          i_left = r1.ntok; i_kstep = r1.kstep; i_vrow = r1.vstride; i_vsafe = r1.v;
-          ikl = r1.k + lane * 16;
-          iv = r1.v + vlane_row * r1.vstride + vlane_ck * 16;
-        }
-      }
-      cp_commit();                                      // one group per call, possibly empty
-      islot = islot + 1 == kStages ? 0 : islot + 1;
-    };
-#pragma unroll
-    for (int i = 0; i < kStages - 1; ++i) issue_next();
-
     // ---- consumer side
-    int cslot = 0;
     for (int cr = 0; cr < nreg; ++cr) {
       const bool thin = cr ? r1.thin : r0.thin;
       const int ntok = cr ? r1.ntok : r0.ntok;
@@ -349,8 +390,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
         cslot = cslot + 1 == kStages ? 0 : cslot + 1;
       }
     }
-    cp_wait<0>();                                       // nothing of this unit is left in flight
-
     // ---- finish the segment: complete unit -> output, otherwise partial state + ticket
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 1);
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
@@ -415,6 +454,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
     }
     f = seg_end;
   }
+  cp_wait<0>();
 }
 
 template <int D, int G>
