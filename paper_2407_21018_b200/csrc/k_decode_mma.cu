@@ -25,10 +25,10 @@ namespace think {
 namespace {
 
 #ifndef THINK_DEC_WARPS
-#define THINK_DEC_WARPS 6
+#define THINK_DEC_WARPS 8
 #endif
 #ifndef THINK_DEC_STAGES
-#define THINK_DEC_STAGES 4
+#define THINK_DEC_STAGES 3
 #endif
 constexpr int kWarps = THINK_DEC_WARPS;  // workers per CTA
 constexpr int kStages = THINK_DEC_STAGES;  // ring depth per warp (kStages - 1 steps in flight)
