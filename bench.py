@@ -125,6 +125,9 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     w = wl.get_config(args.config)
+    if args.lam is not None:
+        import dataclasses
+        w = dataclasses.replace(w, lam=args.lam, name=f"{w.name}-lam{args.lam}")
     nsteps = args.decode_steps if args.decode_steps is not None else w.steps
     cfg = tk.make_config(w.B, w.L, w.N_q, w.N_kv, w.D, w.S_max, w.S_obs, w.recent, nsteps, w.lam, w.torch_dtype)
     cache = tk.ThinKCache(cfg, w.seq_lens, device=dev, keep_scores=True)
@@ -180,12 +183,8 @@ def run_ours(args):
     torch.cuda.synchronize()
     barrier()
     clocks = sampler.stop()
-    total_ms = t_start.elapsed_time(t_end)
-    if world > 1:
-        import torch.distributed as dist
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    from paper_2407_21018_b200 import replicas
+    total_ms, _ = replicas.job_time_and_work(t_start.elapsed_time(t_end), 1.0, device=dev)   # slowest replica
     assert cache.device_error() == 0
 
     prefill_ms = [e["p0"].elapsed_time(e["p1"]) for e in evs]
@@ -239,12 +238,7 @@ def run_ours(args):
             e2e_pass()
         b.record(stream)
         torch.cuda.synchronize()
-        e_ms = a.elapsed_time(b) / n_e2e
-        if world > 1:
-            import torch.distributed as dist
-            tt = torch.tensor([e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e_ms = float(tt.item())
+        e_ms, _ = replicas.job_time_and_work(a.elapsed_time(b) / n_e2e, 1.0, device=dev)
         h2d = sum(x.numel() * x.element_size() for x in (hK, hV, hQ)) + \
             nsteps * sum(v.numel() * v.element_size() for v in hs[0].values())
         d2h = nsteps * hout.numel() * hout.element_size()
@@ -366,6 +360,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--lam", type=float, default=None, help="override the config's pruning ratio (c5 sweep)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
