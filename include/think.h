@@ -203,7 +203,20 @@ thinK_status thinK_score_select_static(const thinK_config* cfg, const int32_t* s
                                        thinK_tensor5 k, int32_t layer0, int32_t nlayers, uint8_t* idx,
                                        double* scores, void* stream);
 
-/* Tokens currently in the unpruned tail of `layer` (S_recent + appended), or -1. */
+/* Periodic re-pruning of the tail (App. C.1 of the paper, without its quantiser): the oldest unpruned
+ * keys are thinned with the channels selected at prefill and joined to the pruned part, so the
+ * full-width tail stops growing over a long generation.  Moves whole blocks of 64 tokens, oldest
+ * first, for as long as at least `keep_recent` tokens stay unpruned; fewer movable tokens than 64 is
+ * not an error (nothing happens).  The values of the moved tokens stay where they are (tail_v).
+ * Attention afterwards treats those tokens like prefix tokens: gathered query x thinned keys.
+ * bf16 caches only (THINK_ERR_UNSUPPORTED otherwise).  All layers of a decode call must have been
+ * re-pruned alike. */
+thinK_status thinK_reprune_tail(thinK_cache* c, int32_t keep_recent, int32_t layer0, int32_t nlayers, void* stream);
+
+/* Tokens of the tail buffers of `layer` whose keys have been re-pruned (a multiple of 64), or -1. */
+int32_t thinK_repruned_len(const thinK_cache* c, int32_t layer);
+
+/* Tokens in the tail buffers of `layer` (S_recent + appended; re-pruned ones included), or -1. */
 int32_t thinK_tail_len(const thinK_cache* c, int32_t layer);
 
 /* Reads the device-side error word (0 = none) with a synchronous copy. */

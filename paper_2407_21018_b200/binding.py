@@ -59,6 +59,8 @@ EXPORTS = {
     "thinK_decode_attn": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_score_select_static": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32), Tensor5, Tensor5, C.c_int32,
                                             C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "thinK_reprune_tail": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_repruned_len": (C.c_int32, [C.c_void_p, C.c_int32]),
     "thinK_tail_len": (C.c_int32, [C.c_void_p, C.c_int32]),
     "thinK_device_error": (C.c_int, [C.c_void_p, C.POINTER(C.c_int32)]),
     "thinK_destroy": (C.c_int, [C.c_void_p]),
@@ -193,6 +195,15 @@ class ThinKCache:
                "thinK_decode_attn")
         return out
 
+    def reprune_tail(self, keep_recent: int, layer0=0, nlayers=None, stream=None):
+        """Thins the oldest whole 64-token blocks of the unpruned tail, keeping >= keep_recent unpruned."""
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        _check(lib.thinK_reprune_tail(self.handle, keep_recent, layer0, nlayers, _stream_ptr(stream)),
+               "thinK_reprune_tail")
+
+    def repruned_len(self, layer=0) -> int:
+        return int(lib.thinK_repruned_len(self.handle, layer))
+
     # -- inspection ------------------------------------------------------
     def tail_len(self, layer=0) -> int:
         return int(lib.thinK_tail_len(self.handle, layer))
@@ -272,7 +283,9 @@ def k_thin_logical(cache: ThinKCache, b: int, l: int, h: int) -> torch.Tensor:
     c = cache.cfg
     S_p = cache.seq_lens[b] - c.S_recent
     nt = [(s - c.S_recent + TILE_TOKENS - 1) // TILE_TOKENS for s in cache.seq_lens]
-    base = sum(c.L * c.N_kv * x for x in nt[:b]) + (l * c.N_kv + h) * nt[b]
+    cap = max(1, c.S_recent + c.max_new_tokens)
+    re_cap = (cap + TILE_TOKENS - 1) // TILE_TOKENS      # tiles reserved per head for re-pruned tail blocks
+    base = sum(c.L * c.N_kv * (x + re_cap) for x in nt[:b]) + (l * c.N_kv + h) * (nt[b] + re_cap)
     flat = cache.k_thin.view(cache.torch_dtype)
     Tp = padded_T(cache.T, c.dtype)
     per = Tp * TILE_TOKENS

@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
   }
   __syncthreads();
 
-  const int64_t gtile = p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * ntiles + tile;
+  const int64_t gtile = p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (ntiles + p.re_cap) + tile;
   uint4* dst = (uint4*)((unsigned char*)p.k_thin + gtile * Tp * kTileTokens * E);
   const int n16 = Tp * kTileTokens * E / 16;
   for (int i = tid; i < n16; i += blockDim.x) dst[i] = ((const uint4*)s_out)[i];
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
   asm volatile("cp.async.wait_group 0;" ::: "memory");
   __syncthreads();
 
-  const int64_t gtile = p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * ntiles + tile;
+  const int64_t gtile = p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (ntiles + p.re_cap) + tile;
   unsigned char* dst = (unsigned char*)p.k_thin + gtile * Tp * 128 + warp * (Tp * 32);   // step = warp
   const int r = lane >> 2, q = lane & 3;
   const unsigned char* rowA = s_in + (warp * 16 + r) * pitch;
@@ -123,6 +123,45 @@ __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
     uint2 v;
     v.x = elem(rowA, c0) | (elem(rowA, c1) << 16);
     v.y = elem(rowB, c0) | (elem(rowB, c1) << 16);
+    *(uint2*)(dst + n16 * 512 + lane * 8) = v;
+  }
+}
+
+// Re-pruning of tail blocks (paper App. C.1: once enough new keys have gathered they are pruned and
+// joined to the pruned part).  One CTA turns one full 64-token tile of the unpruned tail ([D] channels,
+// fragment order) into a thinned tile (the kept channels of idx, fragment order); warp w builds step w.
+__global__ void __launch_bounds__(128) k_reprune_bf16(const RepruneParams p) {
+  const int jt = p.blk0 + blockIdx.x, h = blockIdx.y;
+  const int b = blockIdx.z / p.nlayers, l = p.layer0 + blockIdx.z % p.nlayers;
+  const int lane = threadIdx.x & 31, step = threadIdx.x >> 5;
+  const int D = p.D, T = p.T, Tp = p.Tp;
+  const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+  const int nthin = p.cum_thin[b + 1] - p.cum_thin[b];
+  const unsigned char* src = (const unsigned char*)p.tail_k + (unit * p.tail_tiles_cap + jt) * (int64_t)D * 128;
+  unsigned char* dst = (unsigned char*)p.k_thin +
+                       (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (nthin + p.re_cap) + nthin + jt) * (int64_t)Tp * 128 +
+                       step * (Tp * 32);
+  const uint8_t* ix = p.idx + unit * T;
+  const int r = lane >> 2, q = lane & 3;
+  const int uA = step * 16 + r, uB = uA + 8;
+  auto elem = [&](int u, int c) -> uint32_t {       // kept channel c of token u; channels >= T are padding
+    return c < T ? (uint32_t)*(const uint16_t*)(src + frag_elem_byte(D, ix[c], u)) : 0u;
+  };
+  const int n16 = Tp >> 4;
+  for (int g = 0; g < n16; ++g) {
+    const int c = 16 * g + 2 * q;
+    uint4 v;
+    v.x = elem(uA, c) | (elem(uA, c + 1) << 16);
+    v.y = elem(uA, c + 8) | (elem(uA, c + 9) << 16);
+    v.z = elem(uB, c) | (elem(uB, c + 1) << 16);
+    v.w = elem(uB, c + 8) | (elem(uB, c + 9) << 16);
+    *(uint4*)(dst + g * 512 + lane * 16) = v;
+  }
+  if (Tp & 8) {
+    const int c = 16 * n16 + 2 * q;
+    uint2 v;
+    v.x = elem(uA, c) | (elem(uA, c + 1) << 16);
+    v.y = elem(uB, c) | (elem(uB, c + 1) << 16);
     *(uint2*)(dst + n16 * 512 + lane * 8) = v;
   }
 }
@@ -180,6 +219,12 @@ cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cud
     if (e != cudaSuccess) return e;
     k_compact<float><<<grid, 128, smem, s>>>(p);
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_reprune(const RepruneParams& p, cudaStream_t s) {
+  if (p.nblk <= 0) return cudaSuccess;
+  k_reprune_bf16<<<dim3(p.nblk, p.N_kv, p.B * p.nlayers), 128, 0, s>>>(p);
   return cudaGetLastError();
 }
 

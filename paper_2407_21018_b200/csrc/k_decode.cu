@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(kDecThreads) k_decode_generic(const DecodePara
       int Tc, nvalid;
       if (j < nthin) {
         tile = (const unsigned char*)p.k_thin +
-               (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * nthin + j) * (int64_t)p.T * kTileTokens * E;
+               (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (nthin + p.re_cap) + j) * (int64_t)p.T * kTileTokens * E;
         qs = qs_thin; Tc = p.T;
         nvalid = min(kTileTokens, S_p - j * kTileTokens);
         vrow = (const Tin*)p.v.ptr + b * p.v.sb + (int64_t)j * kTileTokens * p.v.ss + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;

@@ -169,10 +169,20 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       ntiles = je - j0;
       i_kstep = Tp * 32;
       i_vrow = p.v.ss * 2;
-      k0 = (const unsigned char*)p.k_thin + (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * nthin + j0) * (int64_t)Tp * 128;
+      k0 = (const unsigned char*)p.k_thin + (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (nthin + p.re_cap) + j0) * (int64_t)Tp * 128;
       v0 = (const unsigned char*)((const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn) +
            (int64_t)j0 * kTileTokens * i_vrow;
       i_left = min(p.seq_len[b] - p.R, je * kTileTokens) - j0 * kTileTokens;
+    } else if (j0 - nthin < p.n_re) {
+      // tail blocks that were re-pruned: keys thinned like the prefix, values still in the tail buffer
+      const int jb = j0 - nthin, je = min(j1 - nthin, p.n_re);
+      ntiles = je - jb;
+      i_kstep = Tp * 32;
+      i_vrow = D * 2;
+      k0 = (const unsigned char*)p.k_thin +
+           (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (nthin + p.re_cap) + nthin + jb) * (int64_t)Tp * 128;
+      v0 = (const unsigned char*)p.tail_v + (unit_abs * p.cap + (int64_t)jb * kTileTokens) * D * 2;
+      i_left = ntiles * kTileTokens;
     } else {
       const int jb = j0 - nthin, je = j1 - nthin;
       ntiles = je - jb;
@@ -250,37 +260,15 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
     const int64_t unit_abs = ((int64_t)b * p.L + l) * p.N_kv + h;
     const int unit_call = (b * p.nlayers + ll) * p.N_kv + h;
 
-    const unsigned char* kthin = (const unsigned char*)p.k_thin +
-                                 (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * nthin) * (int64_t)Tp * 128;
-    const unsigned char* ktail = (const unsigned char*)p.tail_k + unit_abs * p.tail_tiles_cap * (int64_t)D * 128;
-    const unsigned char* vthin = (const unsigned char*)((const __nv_bfloat16*)p.v.ptr + b * p.v.sb +
-                                                         (int64_t)l * p.v.sl + (int64_t)h * p.v.sn);
-    const unsigned char* vtail = (const unsigned char*)p.tail_v + unit_abs * p.cap * (int64_t)D * 2;
-
-    // ---- the segment is at most two linear streams of 16-token steps: thin tiles, then tail tiles
-    Region r0{}, r1{};
-    int nreg = 0;
-    if (j0 < nthin) {
-      const int je = j1 < nthin ? j1 : nthin;
-      r0.kstep = Tp * 32;
-      r0.k = kthin + (int64_t)j0 * Tp * 128;
-      r0.vstride = p.v.ss * 2;
-      r0.v = vthin + (int64_t)j0 * kTileTokens * r0.vstride;
-      r0.ntok = min(S_p, je * kTileTokens) - j0 * kTileTokens;
-      r0.n16 = n16_thin; r0.has8 = has8_thin; r0.thin = true;
-      nreg = 1;
-    }
+    // ---- the segment is up to three runs of 16-token steps: thin prefix tiles, re-pruned tail blocks
+    // (thin keys as well), unpruned tail tiles.  The consumer only needs their token counts.
+    int seg_ntok[3] = {0, 0, 0};
+    if (j0 < nthin) seg_ntok[0] = min(S_p, (j1 < nthin ? j1 : nthin) * kTileTokens) - j0 * kTileTokens;
     if (j1 > nthin) {
-      Region t;
       const int jb = (j0 > nthin ? j0 : nthin) - nthin, je = j1 - nthin;
-      t.kstep = D * 32;
-      t.k = ktail + (int64_t)jb * D * 128;
-      t.vstride = D * 2;
-      t.v = vtail + (int64_t)jb * kTileTokens * t.vstride;
-      t.ntok = min(p.n_tail, je * kTileTokens) - jb * kTileTokens;
-      t.n16 = KS; t.has8 = false; t.thin = false;
-      if (nreg == 0) r0 = t; else r1 = t;
-      ++nreg;
+      if (jb < p.n_re) seg_ntok[1] = (min(je, p.n_re) - jb) * kTileTokens;
+      const int jb2 = jb > p.n_re ? jb : p.n_re;
+      if (je > jb2) seg_ntok[2] = min(p.n_tail, je * kTileTokens) - jb2 * kTileTokens;
     }
 
     // ---- query fragments (A operand): qa[s][0] = channels 16s+2qd,+1 ; qa[s][1] = channels 16s+2qd+8,+9
@@ -317,10 +305,13 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
     for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
 
     // ---- consumer side
-    for (int cr = 0; cr < nreg; ++cr) {
-      const bool thin = cr ? r1.thin : r0.thin;
-      const int ntok = cr ? r1.ntok : r0.ntok;
-      load_q(thin);
+    int q_kind = -1;                                    // 1: gathered query loaded, 0: full query
+#pragma unroll
+    for (int cr = 0; cr < 3; ++cr) {
+      const int ntok = seg_ntok[cr];
+      if (ntok <= 0) continue;
+      const bool thin = cr < 2;
+      if (q_kind != (int)thin) { load_q(thin); q_kind = thin; }
       const int n16 = thin ? n16_thin : KS;
       const bool has8 = thin && has8_thin;
       for (int left = ntok; left > 0; left -= kStepTokens) {

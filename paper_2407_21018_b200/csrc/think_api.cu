@@ -60,7 +60,7 @@ thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geome
     if (S < c->S_obs || S < c->S_recent || S > c->S_max || S < 1) return THINK_ERR_INVALID_ARG;
     const int nt = (S - c->S_recent + kTileTokens - 1) / kTileTokens;
     g->cum_thin[b + 1] = g->cum_thin[b] + nt;
-    g->thin_tile_base[b + 1] = g->thin_tile_base[b] + (int64_t)c->L * c->N_kv * nt;
+    g->thin_tile_base[b + 1] = g->thin_tile_base[b] + (int64_t)c->L * c->N_kv * (nt + g->tail_tiles_cap);
     if (nt > g->max_thin_tiles) g->max_thin_tiles = nt;
   }
   g->total_thin_tiles = g->thin_tile_base[c->B];
@@ -105,7 +105,8 @@ struct thinK_cache {
   unsigned char* ws;
   void *k_thin, *tail_k, *tail_v, *idx, *scores;
   std::vector<uint8_t> scored, compacted;   // per layer
-  std::vector<int32_t> tail_len;            // per layer, tokens in the tail
+  std::vector<int32_t> tail_len;            // per layer, tokens in the tail buffers
+  std::vector<int32_t> n_re;                // per layer, 64-token tail blocks already re-pruned
   thinK_tensor5 v;                          // borrowed prompt values (set by thinK_compact)
   bool have_v;
   int num_sms, decode_grid_max;
@@ -177,6 +178,7 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
   c->scored.assign(c->g.L, 0);
   c->compacted.assign(c->g.L, 0);
   c->tail_len.assign(c->g.L, 0);
+  c->n_re.assign(c->g.L, 0);
   c->have_v = false;
   int dev = 0;
   cudaDeviceProp prop;
@@ -264,6 +266,7 @@ thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int
   p.idx = (const uint8_t*)c->idx;
   p.k_thin = c->k_thin;
   p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.D = g.D; p.T = g.T; p.Tp = g.Tp; p.R = g.R;
+  p.re_cap = g.tail_tiles_cap;
   p.layer0 = layer0; p.nlayers = nlayers;
   if (launch_compact(p, g.dtype, g.max_thin_tiles, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
   return seed_tail(c, k, v, layer0, nlayers, stream);
@@ -285,7 +288,7 @@ static thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, 
   }
   c->v = v;
   c->have_v = true;
-  for (int l = layer0; l < layer0 + nlayers; ++l) { c->compacted[l] = 1; c->tail_len[l] = g.R; }
+  for (int l = layer0; l < layer0 + nlayers; ++l) { c->compacted[l] = 1; c->tail_len[l] = g.R; c->n_re[l] = 0; }
   return THINK_OK;
 }
 
@@ -329,10 +332,10 @@ thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out)) return THINK_ERR_INVALID_ARG;
   const Geometry& g = c->g;
-  const int n_tail = c->tail_len[layer0];
+  const int n_tail = c->tail_len[layer0], n_re = c->n_re[layer0];
   for (int l = layer0; l < layer0 + nlayers; ++l) {
     if (!c->compacted[l]) return THINK_ERR_STATE;
-    if (c->tail_len[l] != n_tail) return THINK_ERR_STATE;
+    if (c->tail_len[l] != n_tail || c->n_re[l] != n_re) return THINK_ERR_STATE;
   }
   DecodeParams p;
   memset(&p, 0, sizeof(p));
@@ -347,6 +350,8 @@ thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t
   p.counters = (uint32_t*)(c->ws + c->w.decode_counters);
   p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.N_q = g.N_q; p.T = g.T; p.Tp = g.Tp; p.R = g.R; p.cap = g.cap;
   p.tail_tiles_cap = g.tail_tiles_cap;
+  p.re_cap = g.tail_tiles_cap;
+  p.n_re = n_re;
   p.n_tail = n_tail;
   p.n_tail_tiles = (n_tail + kTileTokens - 1) / kTileTokens;
   p.layer0 = layer0; p.nlayers = nlayers;
@@ -356,6 +361,39 @@ thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t
   p.grid = (int)(p.Ntot < (long long)c->decode_grid_max ? p.Ntot : (long long)c->decode_grid_max);
   if (launch_decode(p, g.dtype, g.D, g.G, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
   return THINK_OK;
+}
+
+thinK_status thinK_reprune_tail(thinK_cache* c, int32_t keep_recent, int32_t layer0, int32_t nlayers, void* stream) {
+  if (!c || keep_recent < 0) return THINK_ERR_INVALID_ARG;
+  if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
+  const Geometry& g = c->g;
+  if (g.dtype != THINK_BF16) return THINK_ERR_UNSUPPORTED;
+  const int n_tail = c->tail_len[layer0], n_re = c->n_re[layer0];
+  for (int l = layer0; l < layer0 + nlayers; ++l) {
+    if (!c->compacted[l]) return THINK_ERR_STATE;
+    if (c->tail_len[l] != n_tail || c->n_re[l] != n_re) return THINK_ERR_STATE;
+  }
+  // whole 64-token tiles, oldest first, as long as keep_recent tokens stay unpruned
+  const int movable = n_tail - n_re * kTileTokens - keep_recent;
+  const int nblk = movable > 0 ? movable / kTileTokens : 0;
+  if (nblk == 0) return THINK_OK;
+  RepruneParams p;
+  memset(&p, 0, sizeof(p));
+  p.idx = (const uint8_t*)c->idx;
+  p.thin_tile_base = (const int64_t*)(c->ws + c->w.thin_tile_base);
+  p.cum_thin = (const int32_t*)(c->ws + c->w.cum_thin);
+  p.k_thin = c->k_thin; p.tail_k = c->tail_k;
+  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.D = g.D; p.T = g.T; p.Tp = g.Tp;
+  p.re_cap = g.tail_tiles_cap; p.tail_tiles_cap = g.tail_tiles_cap;
+  p.layer0 = layer0; p.nlayers = nlayers; p.blk0 = n_re; p.nblk = nblk;
+  if (launch_reprune(p, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  for (int l = layer0; l < layer0 + nlayers; ++l) c->n_re[l] = n_re + nblk;
+  return THINK_OK;
+}
+
+int32_t thinK_repruned_len(const thinK_cache* c, int32_t layer) {
+  if (!c || layer < 0 || layer >= c->g.L) return -1;
+  return c->n_re[layer] * kTileTokens;
 }
 
 int32_t thinK_tail_len(const thinK_cache* c, int32_t layer) {

@@ -42,7 +42,19 @@ struct CompactParams {
   const uint8_t* idx;
   void* k_thin;
   int B, L, N_kv, D, T, Tp, R;   // Tp = rows stored per thin tile (T padded to 8 for bf16)
+  int re_cap;                    // tiles reserved per head after the prompt's thin tiles (re-pruned tail blocks)
   int layer0, nlayers;
+};
+
+struct RepruneParams {       // 64-token blocks of the unpruned tail -> thinned tiles (bf16)
+  const uint8_t* idx;
+  const int64_t* thin_tile_base;
+  const int32_t* cum_thin;
+  void* k_thin;
+  const void* tail_k;
+  int B, L, N_kv, D, T, Tp, re_cap, tail_tiles_cap;
+  int layer0, nlayers;
+  int blk0, nblk;           // tail tiles [blk0, blk0 + nblk)
 };
 
 struct TailWriteParams {
@@ -71,7 +83,9 @@ struct DecodeParams {
   uint8_t* records;
   uint32_t* counters;
   int B, L, N_kv, N_q, T, Tp, R, cap, tail_tiles_cap;
-  int n_tail;               // tokens in the tail
+  int re_cap;               // tiles reserved per head after the prompt's thin tiles
+  int n_re;                 // of which hold re-pruned tail blocks (64 tokens each, values stay in tail_v)
+  int n_tail;               // tokens in the tail buffers (re-pruned blocks included)
   int n_tail_tiles;
   int layer0, nlayers;
   long long Ntot;           // tiles over all units of this call
@@ -83,6 +97,7 @@ cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s);
 int score_ctas_per_sm(int dtype, int criterion);
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s);
 cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s);
+cudaError_t launch_reprune(const RepruneParams& p, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int D, int G, cudaStream_t s);
 cudaError_t decode_setup(int dtype, int D, int G);   // one-time per-process kernel attributes
 int decode_workers_per_cta(int dtype);

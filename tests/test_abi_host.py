@@ -49,7 +49,7 @@ def test_cache_bytes_and_memory_model(tk):
     s = tk.thinK_cache_bytes(cfg, [8192])
     T = 76
     n_tiles = math.ceil((8192 - 32) / 64)
-    assert s.k_thin == 32 * 8 * n_tiles * 80 * 64 * 2      # bf16 tiles pad T = 76 to 80 rows
+    assert s.k_thin == 32 * 8 * (n_tiles + 2) * 80 * 64 * 2   # bf16 tiles pad T = 76 to 80 rows; 2 spare tiles per head
     assert s.tail_k == 32 * 8 * math.ceil(96 / 64) * 128 * 64 * 2
     assert s.tail_v == 32 * 8 * 96 * 128 * 2
     assert s.idx == 32 * 8 * T
@@ -74,7 +74,7 @@ def test_ragged_sizes(tk):
     cfg = tk.make_config(3, 2, 4, 4, 64, 128, 32, 32, 8, 0.5, tk.F32)
     s = tk.thinK_cache_bytes(cfg, lens)
     tiles = sum(math.ceil((x - 32) / 64) for x in lens)
-    assert s.k_thin == 2 * 4 * tiles * 32 * 64 * 4
+    assert s.k_thin == 2 * 4 * (tiles + 3 * 1) * 32 * 64 * 4   # one spare tile (cap = 40 tokens) per head and entry
 
 
 @pytest.mark.parametrize("kw", [
