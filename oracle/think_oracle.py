@@ -284,6 +284,21 @@ class ThinKOracle:
                     self.K_full[b][l][h] = np.vstack([self.K_full[b][l][h], np.asarray(k_new[b, l, h], F64)[None]])
                     self.V_all[b][l][h] = np.vstack([self.V_all[b][l][h], np.asarray(v_new[b, l, h], F64)[None]])
 
+    # App. C.1 control flow without the quantiser: prune the oldest unpruned keys, join them to K_T
+    def reprune(self, keep_recent: int, block: int = 64):
+        """Moves whole blocks of `block` tokens, oldest first, from the unpruned keys to the pruned
+        ones (kept channels only, the idx selected at prefill) while >= keep_recent stay unpruned."""
+        for b in range(self.B):
+            for l in range(self.L):
+                for h in range(self.N_kv):
+                    n = self.K_full[b][l][h].shape[0]
+                    m = max(0, (n - keep_recent) // block) * block
+                    if m == 0:
+                        continue
+                    moved = self.K_full[b][l][h][:m][:, self.idx[b, l, h]]
+                    self.K_T[b][l][h] = np.vstack([self.K_T[b][l][h], moved])
+                    self.K_full[b][l][h] = self.K_full[b][l][h][m:]
+
     # decode, steps 6-9
     def decode_attn(self, q: np.ndarray) -> np.ndarray:
         """q [B, L, N_q, D] -> out [B, L, N_q, D]."""

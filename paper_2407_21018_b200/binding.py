@@ -279,7 +279,7 @@ def unpack_tiles(raw: torch.Tensor, n_tiles: int, rows: int, n_tokens: int) -> t
 
 
 def k_thin_logical(cache: ThinKCache, b: int, l: int, h: int) -> torch.Tensor:
-    """Pruned prefix keys of one head as [S_p, T]."""
+    """Pruned keys of one head as [S_p + re-pruned tokens, T]."""
     c = cache.cfg
     S_p = cache.seq_lens[b] - c.S_recent
     nt = [(s - c.S_recent + TILE_TOKENS - 1) // TILE_TOKENS for s in cache.seq_lens]
@@ -290,12 +290,16 @@ def k_thin_logical(cache: ThinKCache, b: int, l: int, h: int) -> torch.Tensor:
     Tp = padded_T(cache.T, c.dtype)
     per = Tp * TILE_TOKENS
     full = unpack_tiles(flat[base * per:(base + nt[b]) * per], nt[b], Tp, S_p)
+    n_re = cache.repruned_len(l) // TILE_TOKENS            # re-pruned tail blocks follow the prompt's tiles
+    if n_re:
+        more = unpack_tiles(flat[(base + nt[b]) * per:(base + nt[b] + n_re) * per], n_re, Tp, n_re * TILE_TOKENS)
+        full = torch.cat([full, more], dim=0)
     assert Tp == cache.T or not full[:, cache.T:].any(), "padding rows of a thin tile must be zero"
     return full[:, :cache.T]
 
 
 def tail_logical(cache: ThinKCache, b: int, l: int, h: int):
-    """Unpruned tail of one head: (keys [n, D], values [n, D])."""
+    """Unpruned tail of one head: (keys [n, D], values [n, D]), re-pruned blocks excluded."""
     c = cache.cfg
     n = cache.tail_len(l)
     cap = max(1, c.S_recent + c.max_new_tokens)
@@ -303,6 +307,7 @@ def tail_logical(cache: ThinKCache, b: int, l: int, h: int):
     unit = (b * c.L + l) * c.N_kv + h
     per = c.D * TILE_TOKENS
     flat = cache.tail_k.view(cache.torch_dtype)
-    keys = unpack_tiles(flat[unit * ttc * per:(unit + 1) * ttc * per], ttc, c.D, n)
-    vals = cache.tail_v.view(cache.torch_dtype)[unit * cap * c.D:(unit * cap + n) * c.D].view(n, c.D)
+    m = cache.repruned_len(l)                              # these tokens now live in k_thin
+    keys = unpack_tiles(flat[unit * ttc * per:(unit + 1) * ttc * per], ttc, c.D, n)[m:]
+    vals = cache.tail_v.view(cache.torch_dtype)[unit * cap * c.D:(unit * cap + n) * c.D].view(n, c.D)[m:]
     return keys, vals

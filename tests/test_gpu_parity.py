@@ -74,6 +74,54 @@ def test_fused_prefill_equals_two_pass_and_repeats():
     assert torch.equal(a.idx_tensor(), c.idx_tensor()) and torch.equal(a.k_thin, c.k_thin)
 
 
+@pytest.mark.parametrize("name,S,R,keep,every", [
+    ("c2", 1000, 32, 32, 40),      # GQA: blocks move at steps 40 and 80 ... while 32 stay unpruned
+    ("c4", 500, 100, 0, 30),       # MHA ragged, T = 51: the recent prompt rows move at once
+    ("c5", 700, 64, 16, 64),
+])
+def test_tail_reprune(name, S, R, keep, every):
+    """thinK_reprune_tail during decode: cache contents bit-exact and attention within tolerance
+    against the oracle that moves the same blocks."""
+    w = dataclasses.replace(wl.shrink(wl.get_config(name), S=S, L=2, B=2, steps=100), S_recent=R)
+    data = wl.make_prefill(w, device="cpu")
+    K, V, Q = data["K"].cuda(), data["V"].cuda(), data["Q_obs"].cuda()
+    cache = make_cache(w, w.steps)
+    cache.prefill(Q, K, V)
+    o = make_oracle(w)
+    o.score_select(to64(data["Q_obs"]), to64(data["K"]))
+    compare_selection(cache.idx_tensor().cpu().numpy(), None, o, w.name)
+    o.compact(to64(data["K"]), to64(data["V"]))
+    moved_any = False
+    for t in range(w.steps):
+        st = wl.make_step(w, t, device="cpu")
+        cache.append(st["k_new"].cuda(), st["v_new"].cuda())
+        o.append(to64(st["k_new"]), to64(st["v_new"]))
+        if t % every == 0:
+            before = cache.repruned_len()
+            cache.reprune_tail(keep)
+            o.reprune(keep)
+            moved_any |= cache.repruned_len() > before
+            assert cache.tail_len() - cache.repruned_len() == o.K_full[0][0][0].shape[0]
+            compare_cache(cache, o, where=f"{w.name} after reprune at step {t}")
+        if t % 7 == 0 or t % every <= 1:
+            out = cache.decode_attn(st["q"].cuda())
+            torch.cuda.synchronize()
+            assert_attn_close(to64(out), o.decode_attn(to64(st["q"])), w.dtype, f"{w.name} step {t}")
+    assert moved_any
+    assert cache.device_error() == 0
+
+
+def test_tail_reprune_rejects_fp32():
+    from paper_2407_21018_b200 import binding as tk
+    w = wl.shrink(wl.get_config("c1"), S=200, steps=2)
+    data = wl.make_prefill(w, device="cuda")
+    c = make_cache(w, 2)
+    c.prefill(data["Q_obs"], data["K"], data["V"])
+    with pytest.raises(tk.ThinKError) as e:
+        c.reprune_tail(0)
+    assert e.value.status == tk.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("lam", [0.0, 0.25, 0.75])
 def test_lambda_sweep(lam):
     w = wl.shrink(wl.get_config("c5"), S=1000, L=1, steps=3, lam=lam)

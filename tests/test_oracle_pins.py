@@ -275,6 +275,45 @@ def test_scale_uses_original_D():
     assert abs(w - 1.0 / (1.0 + math.exp(-a / 2.0))) < 1e-15
 
 
+def test_reprune_makes_recent_tokens_behave_like_prefix_tokens():
+    # A cache built with S_recent = 64 whose 64 recent rows are then re-pruned must equal a cache built
+    # with S_recent = 0 (the score uses all rows either way, so idx is the same); lambda = 0 stays dense.
+    rng = np.random.default_rng(41)
+    B, L, N_q, N_kv, D, S_obs, S = 1, 1, 4, 2, 16, 4, 200
+    K = rng.normal(size=(B, S, L, N_kv, D)) * np.exp(rng.normal(size=D))
+    V = rng.normal(size=(B, S, L, N_kv, D))
+    Q = rng.normal(size=(B, S_obs, L, N_q, D))
+    a = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, 64, 0.5)
+    b = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, 0, 0.5)
+    for o in (a, b):
+        o.score_select(Q, K)
+        o.compact(K, V)
+    assert (a.idx == b.idx).all()
+    a.reprune(keep_recent=0)
+    for h in range(N_kv):
+        assert (a.K_T[0][0][h] == b.K_T[0][0][h]).all() and a.K_full[0][0][h].shape[0] == 0
+    k_new, v_new = rng.normal(size=(B, L, N_kv, D)), rng.normal(size=(B, L, N_kv, D))
+    q = rng.normal(size=(B, L, N_q, D))
+    for o in (a, b):
+        o.append(k_new, v_new)
+    np.testing.assert_allclose(a.decode_attn(q), b.decode_attn(q), rtol=1e-13, atol=1e-14)
+    # keep_recent is honoured and only whole blocks move
+    c = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, 100, 0.5)
+    c.score_select(Q, K)
+    c.compact(K, V)
+    c.reprune(keep_recent=30)            # 100 - 30 = 70 movable -> one block of 64
+    assert c.K_full[0][0][0].shape[0] == 36 and c.K_T[0][0][0].shape[0] == 100 + 64
+    d = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, 100, 0.0)
+    d.score_select(Q, K)
+    d.compact(K, V)
+    d.reprune(keep_recent=0)
+    d.append(k_new, v_new)
+    Kd = np.vstack([K[0, :, 0, 1], k_new[0, 0, 1][None]])
+    Vd = np.vstack([V[0, :, 0, 1], v_new[0, 0, 1][None]])
+    np.testing.assert_allclose(d.decode_attn(q)[0, 0, 2], _dense_by_loops(q[0, 0, 2].tolist(), Kd.tolist(), Vd.tolist()),
+                               rtol=1e-12, atol=1e-13)
+
+
 # ------------------------------------------------------------------ value score (App. D)
 def test_value_score_against_loops():
     rng = np.random.default_rng(21)
