@@ -150,6 +150,8 @@ def run_ours(args):
         for t in range(nsteps):
             s = steps_in[t % nvar]
             cache.append(s["k_new"], s["v_new"])
+            if args.reprune_every and (t + 1) % args.reprune_every == 0:
+                cache.reprune_tail(w.recent)       # App. C.1 control flow: thin the oldest tail blocks
             if ev is not None:
                 ev["d0"][t].record(stream)
             cache.decode_attn(s["q"], out=out)
@@ -360,6 +362,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="c2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--decode-steps", type=int, default=None)
+    ap.add_argument("--reprune-every", type=int, default=0,
+                    help="call thinK_reprune_tail(keep_recent=S_recent) every N decode steps (0 = never); byte "
+                         "accounting stays that of the un-repruned path")
     ap.add_argument("--lam", type=float, default=None, help="override the config's pruning ratio (c5 sweep)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -90,7 +90,7 @@ def shrink(w: Workload, *, S: Optional[int] = None, L: Optional[int] = None, B: 
            steps: Optional[int] = None, lam: Optional[float] = None, name: Optional[str] = None) -> Workload:
     """Same head geometry and law, smaller extent (for parity tests)."""
     B2 = w.B if B is None else B
-    lens = list(w.seq_lens[:B2])
+    lens = [w.seq_lens[i % len(w.seq_lens)] for i in range(B2)]
     if S is not None:
         longest = max(lens)
         # keep the ragged profile: scale every length, never below the window

@@ -22,7 +22,9 @@ def make_cache(w: wl.Workload, steps=None, criterion=0, keep_scores=True):
     steps = w.steps if steps is None else steps
     cfg = tk.make_config(w.B, w.L, w.N_q, w.N_kv, w.D, w.S_max, w.S_obs, w.recent, steps, w.lam,
                          w.torch_dtype, criterion)
-    return tk.ThinKCache(cfg, w.seq_lens, device="cuda", keep_scores=keep_scores)
+    cache = tk.ThinKCache(cfg, w.seq_lens, device="cuda", keep_scores=keep_scores)
+    cache.k_thin.zero_()     # the tiles reserved for re-pruned tail blocks stay unwritten: make buffers comparable
+    return cache
 
 
 def make_oracle(w: wl.Workload) -> orc.ThinKOracle:
