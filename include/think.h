@@ -158,6 +158,31 @@ thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int
 thinK_status thinK_prefill(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0,
                            int32_t nlayers, void* stream);
 
+/* Prefill behind a token-eviction method (the setting of the paper's main experiments, Sec. 4.1-4.2:
+ * H2O or SnapKV first reduce every head to "KV-size" tokens, then the channels of the surviving keys
+ * are pruned).  Instead of gathered K/V tensors the caller passes the method's per-head list of kept
+ * tokens; scoring, compaction and the tail seed read the kept rows straight from the prompt tensors.
+ *   The cache must have been created with seq_lens[b] = n_b, the number of tokens KEPT for entry b
+ *   (the same for every head), and S_max >= max n_b.
+ *   tok:        device int32 [B, L, N_kv, tok_stride]; tok[b][l][h][i], i < n_b, is the row of `k`
+ *               and `v` that holds kept token i of that head.  The order of the list is the token
+ *               order of the compressed cache: its last S_recent entries stay unpruned.  4-byte aligned.
+ *   src_tokens: rows of `k` and `v` per entry; every used tok value must lie in [0, src_tokens).
+ *               The host cannot see the list: an entry outside the range is read as row 0 and sets
+ *               the device error word (thinK_device_error != 0), results are then unspecified.
+ *   q_obs:      as for thinK_score_select (the window's queries are not evicted).
+ *   v_kept:     device buffer of thinK_v_kept_bytes(c); receives the values of the kept tokens as
+ *               dense [B, L, N_kv, S_max, D] and is BORROWED until thinK_destroy (decode reads it);
+ *               `k` and `v` themselves may be released after the call.  One buffer for all layers.
+ * Score[j] sums the squared keys over the kept rows only; everything downstream is thinK_compact
+ * on the gathered tensors.  THINK_ERR_INVALID_ARG if tok_stride < n_b or n_b > src_tokens. */
+thinK_status thinK_prefill_evicted(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v,
+                                   const int32_t* tok, int64_t tok_stride, int32_t src_tokens, void* v_kept,
+                                   int32_t layer0, int32_t nlayers, void* stream);
+
+/* Bytes of the v_kept buffer of thinK_prefill_evicted: B * L * N_kv * S_max * D elements (0 if c is NULL). */
+size_t thinK_v_kept_bytes(const thinK_cache* c);
+
 /* Decode, Sec. 3.3: the new token's key and value join the unpruned tail.
  * k_new, v_new: dense [B, nlayers, N_kv, D].  Every layer of the cache must be
  * appended once per step (any split into layer ranges); THINK_ERR_CAPACITY once

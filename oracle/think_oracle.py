@@ -225,6 +225,27 @@ def think_cache_elements(seq_lens: Sequence[int], L: int, N: int, D: int, keep: 
 
 
 # --------------------------------------------------------------------------
+# Sec. 4.1: ThinK behind a token-eviction method (H2O, SnapKV): that method
+# first reduces every head to "KV-size" tokens; ThinK then prunes the channels
+# of the keys that survived.  The eviction method itself is an input here (a
+# list of kept tokens per head); this routine only forms the compressed tensors
+# that the method would hand over.
+# --------------------------------------------------------------------------
+def gather_kept(X: np.ndarray, tok: np.ndarray, kept: Sequence[int]) -> np.ndarray:
+    """X [B, S, L, N, D], tok [B, L, N, >= kept[b]] (rows of X), kept[b] tokens per head
+    -> [B, max kept, L, N, D] with out[b, i, l, h] = X[b, tok[b, l, h, i], l, h]; rows past
+    kept[b] are NaN (never to be read)."""
+    B, _, L, N, D = X.shape
+    out = np.full((B, max(kept), L, N, D), np.nan, dtype=F64)
+    for b in range(B):
+        for l in range(L):
+            for h in range(N):
+                for i in range(kept[b]):
+                    out[b, i, l, h] = X[b, tok[b, l, h, i], l, h]
+    return out
+
+
+# --------------------------------------------------------------------------
 # The whole path on the paper's B x S x L x N x D tensors, step by step
 # --------------------------------------------------------------------------
 class ThinKOracle:

@@ -55,6 +55,9 @@ EXPORTS = {
     "thinK_score_select": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_compact": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_prefill": (C.c_int, [C.c_void_p, Tensor5, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_prefill_evicted": (C.c_int, [C.c_void_p, Tensor5, Tensor5, Tensor5, C.c_void_p, C.c_int64, C.c_int32,
+                                        C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_v_kept_bytes": (C.c_size_t, [C.c_void_p]),
     "thinK_append": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_decode_attn": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_score_select_static": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32), Tensor5, Tensor5, C.c_int32,
@@ -179,6 +182,20 @@ class ThinKCache:
         self._v = v   # borrowed by the library: keep it alive
         _check(lib.thinK_prefill(self.handle, tensor5(q_obs), tensor5(k), tensor5(v), layer0, nlayers,
                                  _stream_ptr(stream)), "thinK_prefill")
+
+    def prefill_evicted(self, q_obs: Optional[torch.Tensor], k: torch.Tensor, v: torch.Tensor, tok: torch.Tensor,
+                        layer0=0, nlayers=None, stream=None):
+        """Prefill behind a token-eviction method: tok int32 [B, L, N_kv, >= n_b] lists each head's kept rows of
+        k and v (this cache was created with seq_lens = kept counts)."""
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        assert tok.dtype == torch.int32 and tok.dim() == 4 and tok.is_contiguous() and tok.is_cuda
+        assert tuple(tok.shape[:3]) == (self.cfg.B, self.cfg.L, self.cfg.N_kv)
+        if self._v is None:
+            self._v = torch.empty(max(int(lib.thinK_v_kept_bytes(self.handle)), 256), dtype=torch.uint8,
+                                  device=self.device)
+        _check(lib.thinK_prefill_evicted(self.handle, tensor5(q_obs), tensor5(k), tensor5(v), tok.data_ptr(),
+                                         tok.shape[3], k.shape[1], self._v.data_ptr(), layer0, nlayers,
+                                         _stream_ptr(stream)), "thinK_prefill_evicted")
 
     def append(self, k_new: torch.Tensor, v_new: torch.Tensor, layer0=0, nlayers=None, stream=None):
         nlayers = self.cfg.L - layer0 if nlayers is None else nlayers

@@ -38,7 +38,7 @@ __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
   for (int i = tid; i < kTileTokens * cpr; i += blockDim.x) {
     int r = i / cpr, ck = i % cpr;
     uint4 v = make_uint4(0, 0, 0, 0);    // rows past the prefix become zeros
-    if (r < nvalid) v = __ldg((const uint4*)(src + (int64_t)(tok0 + r) * p.k.ss + ck * CH));
+    if (r < nvalid) v = __ldg((const uint4*)(src + token_row(p.tok, unit, tok0 + r) * p.k.ss + ck * CH));
     *(uint4*)(s_in + r * pitch + ck * 16) = v;
   }
   __syncthreads();
@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
   for (int i = tid; i < kTileTokens * cpr; i += 128) {
     const int r = i / cpr, ck = i % cpr;
     const bool ok = r < nvalid;          // rows past the prefix become zeros
-    const void* g = src + (int64_t)(tok0 + (ok ? r : 0)) * p.k.ss + ck * 8;
+    const void* g = src + token_row(p.tok, unit, tok0 + (ok ? r : 0)) * p.k.ss + ck * 8;
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(s_in_addr + r * pitch + ck * 16), "l"(g), "r"(ok ? 16 : 0) : "memory");
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
@@ -182,13 +182,13 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
     int ll = r1 % p.nlayers;
     int b = r1 / p.nlayers;
     int l = p.layer0 + ll;
-    int64_t srow = p.rows_from_seq_len ? (p.seq_len[b] - p.R + r) : r;
+    const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+    int64_t srow = p.rows_from_seq_len ? token_row(p.tok, unit, p.seq_len[b] - p.R + r) : r;
     int sl = l - p.src_layer_base;
     const Tin* ks = (const Tin*)p.k.ptr + b * p.k.sb + srow * p.k.ss + (int64_t)sl * p.k.sl + (int64_t)h * p.k.sn + ck * CH;
     const Tin* vs = (const Tin*)p.v.ptr + b * p.v.sb + srow * p.v.ss + (int64_t)sl * p.v.sl + (int64_t)h * p.v.sn + ck * CH;
     uint4 kv = __ldg((const uint4*)ks);
     uint4 vv = __ldg((const uint4*)vs);
-    const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
     const int u = p.pos0 + r;                       // position in the tail
     *(uint4*)((Tin*)p.tail_v + (unit * p.cap + u) * p.D + ck * CH) = vv;
     unsigned char* tile = (unsigned char*)p.tail_k + (unit * p.tail_tiles_cap + u / kTileTokens) * (int64_t)p.D * kTileTokens * E;
@@ -203,7 +203,38 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
   }
 }
 
+// Values of the kept tokens, gathered into a dense [B, L, N_kv, S_max, D] buffer (token-eviction
+// hook: the decode kernels then read the prefix values from that buffer).  One thread moves 16 bytes.
+template <int E>
+__global__ void __launch_bounds__(256) k_gather_rows(const GatherRowsParams p) {
+  const int cpr = p.D * E / 16;
+  const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.S_max * cpr;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int ck = i % cpr;
+    int64_t r1 = i / cpr;
+    const int t = r1 % p.S_max; r1 /= p.S_max;
+    const int h = r1 % p.N_kv; r1 /= p.N_kv;
+    const int l = p.layer0 + (int)(r1 % p.nlayers);
+    const int b = (int)(r1 / p.nlayers);
+    if (t >= p.seq_len[b]) continue;
+    const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+    const unsigned char* src = (const unsigned char*)p.v.ptr +
+        (b * p.v.sb + token_row(p.tok, unit, t) * p.v.ss + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn) * E + ck * 16;
+    *(uint4*)((unsigned char*)p.dst + ((unit * p.S_max + t) * (int64_t)p.D) * E + ck * 16) = __ldg((const uint4*)src);
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_gather_rows(const GatherRowsParams& p, int dtype, cudaStream_t s) {
+  const int E = dtype == THINK_BF16 ? 2 : 4;
+  const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.S_max * (p.D * E / 16);
+  if (total <= 0) return cudaSuccess;
+  int blocks = (int)((total + 255) / 256 < (int64_t)kSMs * 16 ? (total + 255) / 256 : (int64_t)kSMs * 16);
+  if (E == 2) k_gather_rows<2><<<blocks, 256, 0, s>>>(p);
+  else k_gather_rows<4><<<blocks, 256, 0, s>>>(p);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s) {
   if (max_tiles <= 0) return cudaSuccess;

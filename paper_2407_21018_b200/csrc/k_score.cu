@@ -63,7 +63,7 @@ __device__ void select_head(const double* s, int D, int T, uint8_t* out, int lan
   }
 }
 
-template <typename Tin, bool L1>
+template <typename Tin, bool L1, bool TOK>
 __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const ScoreParams p) {
   constexpr int CH = Chunk<Tin>::CH;
   constexpr bool kBf16 = sizeof(Tin) == 2;
@@ -130,13 +130,15 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
 
   if (active) {
     const Tin* kb = (const Tin*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn + j0;
+    const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+    auto row = [&](int tt) -> int64_t { return TOK ? token_row(p.tok, unit, tt) : (int64_t)tt; };
     int t = t0 + rl;
     const int step = p.RP;
     constexpr int U = 8;
     for (; t + (U - 1) * step < t1; t += U * step) {
       uint4 v[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) v[u] = ldg16(kb + (int64_t)(t + u * step) * p.k.ss);
+      for (int u = 0; u < U; ++u) v[u] = ldg16(kb + row(t + u * step) * p.k.ss);
       if (kBf16) {
         float part[CH];
 #pragma unroll
@@ -164,7 +166,7 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
       }
     }
     for (; t < t1; t += step) {
-      uint4 v = ldg16(kb + (int64_t)t * p.k.ss);
+      uint4 v = ldg16(kb + row(t) * p.k.ss);
       float x[CH];
       Chunk<Tin>::unpack(v, x);
 #pragma unroll
@@ -224,30 +226,33 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
 }  // namespace
 
 // CTAs of the score kernel that are resident per SM (the grid is sized to one wave)
+namespace {
+template <typename Tin, bool L1, bool TOK>
+cudaError_t occupancy_of(int* n) {
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(n, k_colnorm_score_select<Tin, L1, TOK>, kScoreThreads, 0);
+}
+template <typename Tin, bool L1>
+cudaError_t launch_as(const ScoreParams& p, dim3 grid, cudaStream_t s) {
+  if (p.tok.rows) k_colnorm_score_select<Tin, L1, true><<<grid, kScoreThreads, 0, s>>>(p);
+  else k_colnorm_score_select<Tin, L1, false><<<grid, kScoreThreads, 0, s>>>(p);
+  return cudaGetLastError();
+}
+}  // namespace
+
 int score_ctas_per_sm(int dtype, int criterion) {
   int n = 0;
-  cudaError_t e;
   const bool l1 = criterion == THINK_SCORE_KEY_L1;
-  if (dtype == THINK_BF16)
-    e = l1 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_colnorm_score_select<__nv_bfloat16, true>, kScoreThreads, 0)
-           : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_colnorm_score_select<__nv_bfloat16, false>, kScoreThreads, 0);
-  else
-    e = l1 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_colnorm_score_select<float, true>, kScoreThreads, 0)
-           : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_colnorm_score_select<float, false>, kScoreThreads, 0);
+  cudaError_t e;
+  if (dtype == THINK_BF16) e = l1 ? occupancy_of<__nv_bfloat16, true, false>(&n) : occupancy_of<__nv_bfloat16, false, false>(&n);
+  else e = l1 ? occupancy_of<float, true, false>(&n) : occupancy_of<float, false, false>(&n);
   return e == cudaSuccess ? n : 0;
 }
 
 cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s) {
   dim3 grid(p.nsplit, p.ncolblk, p.B * p.nlayers);
   const bool l1 = p.criterion == THINK_SCORE_KEY_L1;
-  if (dtype == THINK_BF16) {
-    if (l1) k_colnorm_score_select<__nv_bfloat16, true><<<grid, kScoreThreads, 0, s>>>(p);
-    else k_colnorm_score_select<__nv_bfloat16, false><<<grid, kScoreThreads, 0, s>>>(p);
-  } else {
-    if (l1) k_colnorm_score_select<float, true><<<grid, kScoreThreads, 0, s>>>(p);
-    else k_colnorm_score_select<float, false><<<grid, kScoreThreads, 0, s>>>(p);
-  }
-  return cudaGetLastError();
+  if (dtype == THINK_BF16) return l1 ? launch_as<__nv_bfloat16, true>(p, grid, s) : launch_as<__nv_bfloat16, false>(p, grid, s);
+  return l1 ? launch_as<float, true>(p, grid, s) : launch_as<float, false>(p, grid, s);
 }
 
 }  // namespace think

@@ -21,7 +21,7 @@ struct Layout {            // byte offsets inside the workspace
 };
 
 struct Geometry {
-  int B, L, N_q, N_kv, D, G, T, Tp, S_obs, R, max_new, cap, tail_tiles_cap, E, dtype, criterion;
+  int B, L, N_q, N_kv, D, G, T, Tp, S_obs, S_max, R, max_new, cap, tail_tiles_cap, E, dtype, criterion;
   int NC, CB, ncolblk, RPmax;
   int64_t total_thin_tiles;    // over all (b, l, h)
   int max_thin_tiles;          // per (l, h) over b
@@ -42,7 +42,7 @@ thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geome
   if (T < 1) return THINK_ERR_INVALID_ARG;
   if ((int64_t)c->B * c->L > 65535) return THINK_ERR_UNSUPPORTED;
   g->B = c->B; g->L = c->L; g->N_q = c->N_q; g->N_kv = c->N_kv; g->D = c->D; g->G = c->N_q / c->N_kv;
-  g->T = T; g->Tp = padded_T(T, c->dtype); g->S_obs = c->S_obs; g->R = c->S_recent; g->max_new = c->max_new_tokens; g->cap = c->S_recent + c->max_new_tokens;
+  g->T = T; g->Tp = padded_T(T, c->dtype); g->S_obs = c->S_obs; g->S_max = c->S_max; g->R = c->S_recent; g->max_new = c->max_new_tokens; g->cap = c->S_recent + c->max_new_tokens;
   if (g->cap < 1) g->cap = 1;
   g->tail_tiles_cap = (g->cap + kTileTokens - 1) / kTileTokens;
   g->dtype = c->dtype; g->E = c->dtype == THINK_BF16 ? 2 : 4; g->criterion = c->criterion;
@@ -210,8 +210,22 @@ static bool layer_range_ok(const thinK_cache* c, int layer0, int nlayers) {
   return layer0 >= 0 && nlayers >= 1 && layer0 + nlayers <= c->g.L;
 }
 
-thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, int32_t layer0,
-                                int32_t nlayers, void* stream) {
+}  // extern "C"
+
+namespace {
+const TokenMap kNoTokenMap = {nullptr, 0, 0, nullptr};
+
+thinK_status make_token_map(thinK_cache* c, const int32_t* tok, int64_t tok_stride, int32_t src_tokens, TokenMap* m) {
+  if (!tok || ((uintptr_t)tok & 3) != 0 || src_tokens < 1) return THINK_ERR_INVALID_ARG;
+  for (int b = 0; b < c->g.B; ++b)
+    if (tok_stride < c->g.seq_len[b] || c->g.seq_len[b] > src_tokens) return THINK_ERR_INVALID_ARG;
+  m->rows = tok; m->stride = tok_stride; m->src_tokens = src_tokens;
+  m->error = (uint32_t*)(c->ws + c->w.error);
+  return THINK_OK;
+}
+
+thinK_status score_select_impl(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, const TokenMap& tok,
+                               int32_t layer0, int32_t nlayers, void* stream) {
   if (!c) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   const Geometry& g = c->g;
@@ -219,6 +233,7 @@ thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tenso
   if (g.criterion == THINK_SCORE_QUERY_DRIVEN && !check_view(q_obs, g.E)) return THINK_ERR_INVALID_ARG;
   ScoreParams p;
   memset(&p, 0, sizeof(p));
+  p.tok = tok;
   p.k = to_view(k);
   p.q = to_view(q_obs);
   p.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
@@ -247,19 +262,23 @@ thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tenso
   return THINK_OK;
 }
 
-static thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int layer0, int nlayers, void* stream);
+thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, const TokenMap& tok, thinK_tensor5 v_prefix,
+                       int layer0, int nlayers, void* stream);
 
-thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0, int32_t nlayers,
-                           void* stream) {
+// `v_prefix`: where decode finds the values of the prefix tokens (the prompt's V itself, or the
+// gathered copy when a token map is in use)
+thinK_status compact_impl(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, const TokenMap& tok, thinK_tensor5 v_prefix,
+                          int32_t layer0, int32_t nlayers, void* stream) {
   if (!c) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   const Geometry& g = c->g;
   if (!check_view(k, g.E) || !check_view(v, g.E)) return THINK_ERR_INVALID_ARG;
   for (int l = layer0; l < layer0 + nlayers; ++l)
     if (!c->scored[l]) return THINK_ERR_STATE;
-  if (c->have_v && memcmp(&c->v, &v, sizeof(v)) != 0) return THINK_ERR_INVALID_ARG;  // one V for all layers
+  if (c->have_v && memcmp(&c->v, &v_prefix, sizeof(v_prefix)) != 0) return THINK_ERR_INVALID_ARG;  // one V for all layers
   CompactParams p;
   memset(&p, 0, sizeof(p));
+  p.tok = tok;
   p.k = to_view(k);
   p.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
   p.thin_tile_base = (const int64_t*)(c->ws + c->w.thin_tile_base);
@@ -269,15 +288,17 @@ thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int
   p.re_cap = g.tail_tiles_cap;
   p.layer0 = layer0; p.nlayers = nlayers;
   if (launch_compact(p, g.dtype, g.max_thin_tiles, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
-  return seed_tail(c, k, v, layer0, nlayers, stream);
+  return seed_tail(c, k, v, tok, v_prefix, layer0, nlayers, stream);
 }
 
 // seeds the unpruned tail with the last S_recent prompt rows (keys and values) and books the layers
-static thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int layer0, int nlayers, void* stream) {
+thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, const TokenMap& tok, thinK_tensor5 v_prefix,
+                       int layer0, int nlayers, void* stream) {
   const Geometry& g = c->g;
   if (g.R > 0) {
     TailWriteParams t;
     memset(&t, 0, sizeof(t));
+    t.tok = tok;
     t.k = to_view(k); t.v = to_view(v);
     t.src_layer_base = 0; t.rows_from_seq_len = 1;
     t.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
@@ -286,10 +307,57 @@ static thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, 
     t.layer0 = layer0; t.nlayers = nlayers; t.nrows = g.R; t.pos0 = 0;
     if (launch_tail_write(t, g.dtype, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
   }
-  c->v = v;
+  c->v = v_prefix;
   c->have_v = true;
   for (int l = layer0; l < layer0 + nlayers; ++l) { c->compacted[l] = 1; c->tail_len[l] = g.R; c->n_re[l] = 0; }
   return THINK_OK;
+}
+}  // namespace
+
+extern "C" {
+
+thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, int32_t layer0,
+                                int32_t nlayers, void* stream) {
+  return score_select_impl(c, q_obs, k, kNoTokenMap, layer0, nlayers, stream);
+}
+
+thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0, int32_t nlayers,
+                           void* stream) {
+  return compact_impl(c, k, v, kNoTokenMap, v, layer0, nlayers, stream);
+}
+
+size_t thinK_v_kept_bytes(const thinK_cache* c) {
+  if (!c) return 0;
+  const Geometry& g = c->g;
+  return (size_t)g.B * g.L * g.N_kv * g.S_max * g.D * g.E;
+}
+
+thinK_status thinK_prefill_evicted(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v,
+                                   const int32_t* tok, int64_t tok_stride, int32_t src_tokens, void* v_kept,
+                                   int32_t layer0, int32_t nlayers, void* stream) {
+  if (!c || !v_kept || !aligned16(v_kept)) return THINK_ERR_INVALID_ARG;
+  if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
+  const Geometry& g = c->g;
+  if (!check_view(v, g.E)) return THINK_ERR_INVALID_ARG;
+  TokenMap m;
+  thinK_status st = make_token_map(c, tok, tok_stride, src_tokens, &m);
+  if (st != THINK_OK) return st;
+  st = score_select_impl(c, q_obs, k, m, layer0, nlayers, stream);
+  if (st != THINK_OK) return st;
+  // values of the kept tokens: dense [B, L, N_kv, S_max, D]
+  GatherRowsParams gp;
+  memset(&gp, 0, sizeof(gp));
+  gp.tok = m; gp.v = to_view(v);
+  gp.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
+  gp.dst = v_kept;
+  gp.B = g.B; gp.L = g.L; gp.N_kv = g.N_kv; gp.D = g.D; gp.S_max = g.S_max;
+  gp.layer0 = layer0; gp.nlayers = nlayers;
+  if (launch_gather_rows(gp, g.dtype, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  thinK_tensor5 vk;
+  vk.ptr = v_kept;
+  vk.stride_s = g.D; vk.stride_n = (int64_t)g.S_max * g.D; vk.stride_l = (int64_t)g.N_kv * vk.stride_n;
+  vk.stride_b = (int64_t)g.L * vk.stride_l;
+  return compact_impl(c, k, v, m, vk, layer0, nlayers, stream);
 }
 
 thinK_status thinK_prefill(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0,

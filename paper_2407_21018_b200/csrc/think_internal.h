@@ -20,7 +20,19 @@ struct View5 {
   int64_t sb, ss, sl, sn;   // element strides
 };
 
+// Optional token-eviction hook: kept token i of unit (b, l, h) is row rows[unit * stride + i] of the
+// source views.  rows == nullptr means the identity (row i).  Entries outside [0, src_tokens) set the
+// error word and are read as row 0.
+struct TokenMap {
+  const int32_t* rows;
+  int64_t stride;
+  int32_t src_tokens;
+  uint32_t* error;
+};
+constexpr uint32_t kErrTokenRange = 1u;   // device error word: a token index was out of range
+
 struct ScoreParams {
+  TokenMap tok;
   View5 k, q;
   const int32_t* seq_len;
   double* partials;
@@ -36,6 +48,7 @@ struct ScoreParams {
 };
 
 struct CompactParams {
+  TokenMap tok;
   View5 k;
   const int32_t* seq_len;
   const int64_t* thin_tile_base;
@@ -57,7 +70,17 @@ struct RepruneParams {       // 64-token blocks of the unpruned tail -> thinned 
   int blk0, nblk;           // tail tiles [blk0, blk0 + nblk)
 };
 
+struct GatherRowsParams {    // values of the kept tokens -> dense [B, L, N_kv, S_max, D]
+  TokenMap tok;
+  View5 v;
+  const int32_t* seq_len;
+  void* dst;
+  int B, L, N_kv, D, S_max;
+  int layer0, nlayers;
+};
+
 struct TailWriteParams {
+  TokenMap tok;             // applies when rows_from_seq_len is set
   View5 k, v;               // sources
   int src_layer_base;       // layer index subtracted before applying sl
   int rows_from_seq_len;    // 1: source row = seq_len[b] - R + r ; 0: source row = r
@@ -98,6 +121,7 @@ int score_ctas_per_sm(int dtype, int criterion);
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s);
 cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_reprune(const RepruneParams& p, cudaStream_t s);
+cudaError_t launch_gather_rows(const GatherRowsParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int D, int G, cudaStream_t s);
 cudaError_t decode_setup(int dtype, int D, int G);   // one-time per-process kernel attributes
 int decode_workers_per_cta(int dtype);
@@ -132,6 +156,17 @@ __host__ __device__ __forceinline__ int frag_elem_byte(int Cp, int c, int u) {
   }
   const int w = c - n16 * 16, q = w >> 1, lo = w & 1;
   return base + n16 * 512 + (r * 4 + q) * 8 + jx * 4 + lo * 2;
+}
+
+// source row of kept token i of `unit`
+__device__ __forceinline__ int64_t token_row(const TokenMap& m, int64_t unit, int i) {
+  if (!m.rows) return i;
+  const int32_t r = __ldg(m.rows + unit * m.stride + i);
+  if ((uint32_t)r >= (uint32_t)m.src_tokens) {
+    atomicOr(m.error, kErrTokenRange);
+    return 0;
+  }
+  return r;
 }
 
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }

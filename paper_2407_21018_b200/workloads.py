@@ -23,7 +23,7 @@ from typing import List, Optional, Tuple
 
 import torch
 
-__all__ = ["Workload", "CONFIGS", "get_config", "shrink", "make_prefill", "make_step"]
+__all__ = ["Workload", "CONFIGS", "get_config", "shrink", "make_prefill", "make_step", "make_eviction", "evicted"]
 
 
 @dataclasses.dataclass(frozen=True)
@@ -98,6 +98,34 @@ def shrink(w: Workload, *, S: Optional[int] = None, L: Optional[int] = None, B: 
     return dataclasses.replace(
         w, name=name or (w.name + "-small"), B=B2, L=w.L if L is None else L, seq_lens=tuple(lens),
         steps=w.steps if steps is None else steps, lam=w.lam if lam is None else lam)
+
+
+def evicted(w: Workload, kv_sizes) -> Workload:
+    """The workload a cache sees behind a token-eviction method that kept kv_sizes[b] tokens per head."""
+    if isinstance(kv_sizes, int):
+        kv_sizes = (kv_sizes,) * w.B
+    assert len(kv_sizes) == w.B and all(w.recent <= n <= s and w.S_obs <= n for n, s in zip(kv_sizes, w.seq_lens))
+    return dataclasses.replace(w, name=w.name + "-evicted", seq_lens=tuple(int(n) for n in kv_sizes))
+
+
+def make_eviction(w: Workload, kv_sizes, device="cpu") -> torch.Tensor:
+    """Stand-in for the output of an upstream token-eviction method (H2O / SnapKV style): for every
+    (b, l, h) the observation window (last S_obs prompt rows) plus a seeded random subset of the earlier
+    rows, kv_sizes[b] rows in all, ascending.  int32 [B, L, N_kv, max kv_size]; unused slots hold -1."""
+    if isinstance(kv_sizes, int):
+        kv_sizes = (kv_sizes,) * w.B
+    width = max(kv_sizes)
+    tok = torch.full((w.B, w.L, w.N_kv, width), -1, dtype=torch.int32)
+    for b in range(w.B):
+        S_b, n = w.seq_lens[b], int(kv_sizes[b])
+        assert w.S_obs <= n <= S_b
+        early = S_b - w.S_obs
+        key = torch.rand((w.L, w.N_kv, max(early, 1)), generator=_gen("cpu", w.seed, 9, b))
+        pick = torch.topk(key, n - w.S_obs, dim=-1).indices.sort(dim=-1).values if n > w.S_obs else \
+            torch.empty((w.L, w.N_kv, 0), dtype=torch.int64)
+        window = torch.arange(early, S_b).expand(w.L, w.N_kv, w.S_obs)
+        tok[b, :, :, :n] = torch.cat([pick, window], dim=-1).to(torch.int32)
+    return tok.to(device)
 
 
 def _gen(device, seed: int, *ids: int) -> torch.Generator:

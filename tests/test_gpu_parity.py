@@ -122,6 +122,73 @@ def test_tail_reprune_rejects_fp32():
     assert e.value.status == tk.ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("name,S,kv,R", [
+    ("c2", 1500, 256, 32),                     # GQA bf16, the paper's KV-size range (128..2048)
+    ("c2", 900, 128, 0),                       # no recent window: everything thinned
+    ("c4", 700, (130, 257, 64), 32),           # MHA, ragged prompts and ragged kept counts, T = 51
+    ("c1", 300, 100, 32),                      # fp32 kernels
+])
+def test_prefill_behind_token_eviction(name, S, kv, R):
+    """thinK_prefill_evicted with a per-head list of kept tokens equals the oracle run on the tensors
+    an eviction method would hand over (each head's kept rows gathered)."""
+    base = wl.get_config(name)
+    B = len(kv) if isinstance(kv, tuple) else min(base.B, 2)
+    src = dataclasses.replace(wl.shrink(base, S=S, L=min(base.L, 2), B=B, steps=4), S_recent=R)
+    data = wl.make_prefill(src, device="cpu")
+    tok = wl.make_eviction(src, kv)
+    w = wl.evicted(src, kv)
+    cache = make_cache(w, w.steps)
+    cache.prefill_evicted(data["Q_obs"].cuda(), data["K"].cuda(), data["V"].cuda(), tok.cuda())
+    torch.cuda.synchronize()
+    assert cache.device_error() == 0
+    o = make_oracle(w)
+    tok64 = tok.numpy().astype(np.int64)
+    Kg = orc.gather_kept(to64(data["K"]), tok64, list(w.seq_lens))
+    Vg = orc.gather_kept(to64(data["V"]), tok64, list(w.seq_lens))
+    o.score_select(to64(data["Q_obs"]), Kg)
+    compare_selection(cache.idx_tensor().cpu().numpy(), cache.scores_tensor().cpu().numpy(), o, w.name)
+    o.compact(Kg, Vg)
+    compare_cache(cache, o, where=w.name)
+    for t in range(w.steps):
+        st = wl.make_step(w, t, device="cpu")
+        cache.append(st["k_new"].cuda(), st["v_new"].cuda())
+        out = cache.decode_attn(st["q"].cuda())
+        torch.cuda.synchronize()
+        o.append(to64(st["k_new"]), to64(st["v_new"]))
+        assert_attn_close(to64(out), o.decode_attn(to64(st["q"])), w.dtype, f"{w.name} step {t}")
+    assert cache.device_error() == 0
+
+
+def test_eviction_list_out_of_range_is_flagged():
+    """A kept-token entry outside the source rows is never dereferenced: it is read as row 0 and the
+    device error word is set."""
+    src = wl.shrink(wl.get_config("c2"), S=400, L=1, steps=1)
+    data = wl.make_prefill(src, device="cuda")
+    tok = wl.make_eviction(src, 128)
+    tok[0, 0, 3, 5] = 400                      # one past the last source row
+    w = wl.evicted(src, 128)
+    cache = make_cache(w, 1)
+    cache.prefill_evicted(data["Q_obs"], data["K"], data["V"], tok.cuda())
+    torch.cuda.synchronize()
+    assert cache.device_error() != 0
+
+
+def test_eviction_rejects_bad_arguments():
+    from paper_2407_21018_b200 import binding as tk
+    src = wl.shrink(wl.get_config("c2"), S=400, L=1, steps=1)
+    data = wl.make_prefill(src, device="cuda")
+    w = wl.evicted(src, 128)
+    cache = make_cache(w, 1)
+    short = wl.make_eviction(src, 128)[..., :100].contiguous().cuda()     # list shorter than the kept count
+    with pytest.raises(tk.ThinKError) as e:
+        cache.prefill_evicted(data["Q_obs"], data["K"], data["V"], short)
+    assert e.value.status == tk.ERR_INVALID_ARG
+    tok = wl.make_eviction(src, 128).cuda()
+    with pytest.raises(tk.ThinKError) as e:                                # source with fewer rows than kept
+        cache.prefill_evicted(data["Q_obs"], data["K"][:, :100], data["V"][:, :100], tok)
+    assert e.value.status == tk.ERR_INVALID_ARG
+
+
 @pytest.mark.parametrize("lam", [0.0, 0.25, 0.75])
 def test_lambda_sweep(lam):
     w = wl.shrink(wl.get_config("c5"), S=1000, L=1, steps=3, lam=lam)

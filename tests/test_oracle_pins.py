@@ -314,6 +314,51 @@ def test_reprune_makes_recent_tokens_behave_like_prefix_tokens():
                                rtol=1e-12, atol=1e-13)
 
 
+# ------------------------------------------------------------------ behind a token-eviction method (Sec. 4.1)
+def test_eviction_equals_masking_the_evicted_tokens():
+    # Evicting a token from a head is the same as that token never receiving attention: with the evicted
+    # key rows set to zero the literal Frobenius score is unchanged (zero rows add nothing), and dense
+    # attention over the kept rows only must equal the path with lambda = 0 on the gathered tensors.
+    rng = np.random.default_rng(77)
+    B, L, N_q, N_kv, D, S_obs, S, n = 1, 2, 4, 2, 12, 3, 40, 17
+    K = rng.normal(size=(B, S, L, N_kv, D)) * np.exp(rng.normal(size=D))
+    V = rng.normal(size=(B, S, L, N_kv, D))
+    Q = rng.normal(size=(B, S_obs, L, N_q, D))
+    tok = np.zeros((B, L, N_kv, n), dtype=np.int64)
+    for l in range(L):
+        for h in range(N_kv):
+            early = np.sort(rng.permutation(S - S_obs)[: n - S_obs])
+            tok[0, l, h] = np.concatenate([early, np.arange(S - S_obs, S)])
+    Kg, Vg = orc.gather_kept(K, tok, [n]), orc.gather_kept(V, tok, [n])
+    assert Kg.shape == (B, n, L, N_kv, D)
+    o = orc.ThinKOracle(B, L, N_q, N_kv, D, [n], S_obs, S_obs, 0.5)
+    o.score_select(Q, Kg)
+    for l in range(L):
+        for h in range(N_kv):
+            mask = np.zeros(S)
+            mask[tok[0, l, h]] = 1.0
+            Qg = np.stack([Q[0, :, l, h * 2 + g] for g in range(2)])
+            want = orc.score_literal(Qg, K[0, :, l, h] * mask[:, None])
+            np.testing.assert_allclose(o.score[0, l, h], want, rtol=1e-12)
+            # different heads keep different tokens, and the gather follows each head's own list
+            assert (Kg[0, :, l, h] == K[0, tok[0, l, h], l, h]).all()
+    assert (tok[0, 0, 0] != tok[0, 0, 1]).any()
+    d = orc.ThinKOracle(B, L, N_q, N_kv, D, [n], S_obs, S_obs, 0.0)
+    d.score_select(Q, Kg)
+    d.compact(Kg, Vg)
+    q = rng.normal(size=(B, L, N_q, D))
+    out = d.decode_attn(q)
+    for l in range(L):
+        for hq in range(N_q):
+            h = hq // 2
+            rows = tok[0, l, h].tolist()
+            want = _dense_by_loops(q[0, l, hq].tolist(), K[0, rows, l, h].tolist(), V[0, rows, l, h].tolist())
+            np.testing.assert_allclose(out[0, l, hq], want, rtol=1e-12, atol=1e-13)
+    # identity list = no eviction
+    ident = np.broadcast_to(np.arange(S), (B, L, N_kv, S))
+    assert (orc.gather_kept(K, ident, [S]) == K).all()
+
+
 # ------------------------------------------------------------------ value score (App. D)
 def test_value_score_against_loops():
     rng = np.random.default_rng(21)
