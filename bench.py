@@ -50,6 +50,13 @@ def prefill_bytes(w: wl.Workload, T: int) -> int:
     return tot
 
 
+def prefill_bytes_evicted(w: wl.Workload, T: int) -> int:
+    """Same behind a token-eviction method (`w` = the workload after eviction, seq_lens = kept tokens):
+    the kept key rows and their list are read once, the kept value rows are read and written once."""
+    e = w.elem_bytes
+    return prefill_bytes(w, T) + sum(S * 4 + 2 * (S - w.recent) * w.D * e for S in w.seq_lens) * w.L * w.N_kv
+
+
 def decode_bytes(w: wl.Workload, T: int, t: int) -> int:
     """Algorithmic bytes of decode step t (t tokens already appended before it): thinned prefix
     keys, unpruned tail keys, all values, index list, q in and out."""
@@ -129,11 +136,19 @@ def run_ours(args):
         import dataclasses
         w = dataclasses.replace(w, lam=args.lam, name=f"{w.name}-lam{args.lam}")
     nsteps = args.decode_steps if args.decode_steps is not None else w.steps
+    tok = None
+    if args.kv_size:
+        # Sec. 4.1 setting: an upstream eviction method kept kv_size tokens per head; the cache holds those
+        src = w
+        tok = wl.make_eviction(src, args.kv_size).to(dev)
+        w = wl.evicted(src, args.kv_size)
+        data = wl.make_prefill(src, device=dev, pad_nan=False)
+    else:
+        data = wl.make_prefill(w, device=dev, pad_nan=False)
     cfg = tk.make_config(w.B, w.L, w.N_q, w.N_kv, w.D, w.S_max, w.S_obs, w.recent, nsteps, w.lam, w.torch_dtype)
     cache = tk.ThinKCache(cfg, w.seq_lens, device=dev, keep_scores=True)
     T = cache.T
 
-    data = wl.make_prefill(w, device=dev, pad_nan=False)
     K, V, Q = data["K"], data["V"], data["Q_obs"]
     nvar = min(4, max(1, nsteps))
     steps_in = [wl.make_step(w, t, device=dev) for t in range(nvar)]
@@ -143,8 +158,11 @@ def run_ours(args):
     def one_pass(ev=None):
         if ev is not None:
             ev["p0"].record(stream)
-        cache.score_select(Q, K)
-        cache.compact(K, V)
+        if tok is not None:
+            cache.prefill_evicted(Q, K, V, tok)
+        else:
+            cache.score_select(Q, K)
+            cache.compact(K, V)
         if ev is not None:
             ev["p1"].record(stream)
         for t in range(nsteps):
@@ -194,7 +212,7 @@ def run_ours(args):
     dec_mean_us = 1e3 * sum(sum(r) for r in dec_ms) / max(1, args.steps * nsteps)
     dec_bytes = [decode_bytes(w, T, t) for t in range(nsteps)]
     dec_bytes_mean = sum(dec_bytes) / max(1, nsteps)
-    pre_b = prefill_bytes(w, T)
+    pre_b = prefill_bytes_evicted(w, T) if tok is not None else prefill_bytes(w, T)
     pre_us = 1e3 * sum(prefill_ms) / len(prefill_ms)
     pass_bytes = pre_b + sum(dec_bytes) + nsteps * append_bytes(w)
     ms_per_step = total_ms / args.steps
@@ -221,8 +239,11 @@ def run_ours(args):
             K.copy_(hK, non_blocking=True)
             V.copy_(hV, non_blocking=True)
             Q.copy_(hQ, non_blocking=True)
-            cache.score_select(Q, K)
-            cache.compact(K, V)
+            if tok is not None:
+                cache.prefill_evicted(Q, K, V, tok)
+            else:
+                cache.score_select(Q, K)
+                cache.compact(K, V)
             for t in range(nsteps):
                 s = hs[t % nvar]
                 dq.copy_(s["q"], non_blocking=True)
@@ -275,7 +296,8 @@ def run_ours(args):
                          "traffic": NCU_DECODE_TRAFFIC_BYTES.get(w.name), "traffic_unit": "bytes per launch"},
             "clocks": clocks,
             "e2e": e2e,
-            "gpu_launches": args.steps * (2 + (1 if w.recent > 0 else 0) + 2 * nsteps),
+            "gpu_launches": args.steps * (2 + (1 if w.recent > 0 else 0) + (1 if tok is not None else 0) + 2 * nsteps
+                                          + (nsteps // args.reprune_every if args.reprune_every else 0)),
             "cpu_baseline": cpu,
         }
         print(json.dumps(line))
@@ -365,6 +387,9 @@ def main():
     ap.add_argument("--reprune-every", type=int, default=0,
                     help="call thinK_reprune_tail(keep_recent=S_recent) every N decode steps (0 = never); byte "
                          "accounting stays that of the un-repruned path")
+    ap.add_argument("--kv-size", type=int, default=0,
+                    help="prefill behind a token-eviction method that kept this many tokens per head "
+                         "(thinK_prefill_evicted on seeded kept-token lists); 0 = no eviction")
     ap.add_argument("--lam", type=float, default=None, help="override the config's pruning ratio (c5 sweep)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -10,7 +10,8 @@ namespace {
 // One CTA builds one tile: 64 token rows of one head are staged in shared memory (padded pitch),
 // the threads gather the kept channels into the tile image in shared memory, and the finished
 // image leaves with coalesced 16-byte stores.
-template <typename Tin>
+// TOK: rows come from a per-head kept-token list (token-eviction hook) instead of the prompt order.
+template <typename Tin, bool TOK>
 __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
   constexpr int E = sizeof(Tin);
   constexpr int CH = 16 / E;             // elements per 16-byte chunk
@@ -38,7 +39,10 @@ __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
   for (int i = tid; i < kTileTokens * cpr; i += blockDim.x) {
     int r = i / cpr, ck = i % cpr;
     uint4 v = make_uint4(0, 0, 0, 0);    // rows past the prefix become zeros
-    if (r < nvalid) v = __ldg((const uint4*)(src + token_row(p.tok, unit, tok0 + r) * p.k.ss + ck * CH));
+    if (r < nvalid) {
+      const int64_t row = TOK ? token_row(p.tok, unit, tok0 + r) : (int64_t)(tok0 + r);
+      v = __ldg((const uint4*)(src + row * p.k.ss + ck * CH));
+    }
     *(uint4*)(s_in + r * pitch + ck * 16) = v;
   }
   __syncthreads();
@@ -67,6 +71,7 @@ __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
 // flight at once); then warp w builds the four 16-token steps w of the tile: for each group of 16
 // kept channels a lane gathers the eight elements of its 16-byte fragment piece (two tokens x four
 // channels) and the warp writes the 512-byte chunk straight to global memory.
+template <bool TOK>
 __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
   const int D = p.D, T = p.T, Tp = p.Tp;
@@ -92,7 +97,8 @@ __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
   for (int i = tid; i < kTileTokens * cpr; i += 128) {
     const int r = i / cpr, ck = i % cpr;
     const bool ok = r < nvalid;          // rows past the prefix become zeros
-    const void* g = src + token_row(p.tok, unit, tok0 + (ok ? r : 0)) * p.k.ss + ck * 8;
+    const int64_t row = TOK ? token_row(p.tok, unit, tok0 + (ok ? r : 0)) : (int64_t)(tok0 + (ok ? r : 0));
+    const void* g = src + row * p.k.ss + ck * 8;
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(s_in_addr + r * pitch + ck * 16), "l"(g), "r"(ok ? 16 : 0) : "memory");
   }
   asm volatile("cp.async.commit_group;" ::: "memory");
@@ -244,11 +250,16 @@ cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cud
   cudaError_t e;
   if (dtype == THINK_BF16) {
     smem = (size_t)kTileTokens * (p.D * 2 + 16) + ((p.Tp + 15) & ~15);
-    k_compact_bf16<<<grid, 128, smem, s>>>(p);
-  } else {
-    e = cudaFuncSetAttribute(k_compact<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (p.tok.rows) k_compact_bf16<true><<<grid, 128, smem, s>>>(p);
+    else k_compact_bf16<false><<<grid, 128, smem, s>>>(p);
+  } else if (p.tok.rows) {
+    e = cudaFuncSetAttribute(k_compact<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    k_compact<float><<<grid, 128, smem, s>>>(p);
+    k_compact<float, true><<<grid, 128, smem, s>>>(p);
+  } else {
+    e = cudaFuncSetAttribute(k_compact<float, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    k_compact<float, false><<<grid, 128, smem, s>>>(p);
   }
   return cudaGetLastError();
 }
