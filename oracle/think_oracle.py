@@ -24,6 +24,11 @@ What the paper fixes and what it leaves open
   the two logit vectors are concatenated, scaled by 1/sqrt(D) with the
   original D, and go through ONE softmax; the value cache is untouched.
 
+* Value-channel pruning (App. D): Score_v = column norms of the window's
+  attention output, top-T_v kept.  App. D stops at the criterion; carrying it
+  through decode like the keys (prefix rows thinned, recent and new rows whole,
+  a pruned prefix channel counting as zero) is a declared reading.
+
 Pins (tests/test_oracle_pins.py): rank-one Frobenius identity, Eq. 2's loss for
 one pruned channel, brute-force subset search, lambda = 0 and S_recent = S
 reducing to dense attention computed by a separately written routine, hand
@@ -201,6 +206,24 @@ def score_value(Q_obs: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarray:
     return np.sqrt(np.sum(O * O, axis=0))
 
 
+def decode_attention_kv(q: np.ndarray, K_T: np.ndarray, idx: np.ndarray, K_full: np.ndarray, V_T: np.ndarray,
+                        idx_v: np.ndarray, V_full: np.ndarray) -> np.ndarray:
+    """App. D carried through decode the way Sec. 3.3 treats the keys (declared reading: App. D gives
+    the criterion only): the values of the pruned prefix keep T_v channels, V_T [S_p, T_v] with kept
+    channels idx_v; recent and decoded tokens keep full rows, V_full [U, D].  The attention weights are
+    those of decode_attention; a pruned value channel of a prefix token counts as zero, so the output
+    channel j sums the tail's share everywhere and the prefix's share only where j is kept."""
+    q = np.asarray(q, dtype=F64)
+    D = q.shape[0]
+    x_p = np.asarray(K_T, dtype=F64) @ q[idx]
+    x_r = np.asarray(K_full, dtype=F64) @ q
+    p = _softmax(np.concatenate([x_p, x_r]) / math.sqrt(D))
+    S_p = x_p.shape[0]
+    out = p[S_p:] @ np.asarray(V_full, dtype=F64)
+    out[idx_v] += p[:S_p] @ np.asarray(V_T, dtype=F64)
+    return out
+
+
 # --------------------------------------------------------------------------
 # Sec. 3.1 cache-size model and the Table 7 accounting
 # --------------------------------------------------------------------------
@@ -253,7 +276,7 @@ class ThinKOracle:
     (batch entry, layer, key head), with the per-head routines above."""
 
     def __init__(self, B: int, L: int, N_q: int, N_kv: int, D: int, seq_lens: Sequence[int], S_obs: int,
-                 S_recent: int, lam: float):
+                 S_recent: int, lam: float, lam_v: float = 0.0):
         assert N_q % N_kv == 0
         self.B, self.L, self.N_q, self.N_kv, self.D = B, L, N_q, N_kv, D
         self.G = N_q // N_kv
@@ -262,6 +285,11 @@ class ThinKOracle:
         self.T = kept_channels(lam, D)
         self.idx = None
         self.score = None
+        # App. D: value channels are pruned too when lam_v > 0
+        self.lam_v = lam_v
+        self.T_v = kept_channels(lam_v, D)
+        self.idx_v = None
+        self.score_v = None
 
     # prefill, steps 1-3
     def score_select(self, Q_obs: np.ndarray, K: np.ndarray, literal: bool = False):
@@ -280,6 +308,21 @@ class ThinKOracle:
                     self.idx[b, l, h] = select_top_T(s, self.T)
         return self.idx
 
+    # App. D Eqs. 3-4: value-channel scores and their top-T_v
+    def score_select_v(self, Q_obs: np.ndarray, K: np.ndarray, V: np.ndarray):
+        B, L, N_kv, D, G = self.B, self.L, self.N_kv, self.D, self.G
+        self.idx_v = np.zeros((B, L, N_kv, self.T_v), dtype=np.int64)
+        self.score_v = np.zeros((B, L, N_kv, D), dtype=F64)
+        for b in range(B):
+            S_b = self.seq_lens[b]
+            for l in range(L):
+                for h in range(N_kv):
+                    Qg = np.stack([Q_obs[b, :, l, h * G + g, :] for g in range(G)])
+                    s = score_value(Qg, K[b, :S_b, l, h, :], V[b, :S_b, l, h, :])
+                    self.score_v[b, l, h] = s
+                    self.idx_v[b, l, h] = select_top_T(s, self.T_v)
+        return self.idx_v
+
     # prefill, step 4
     def compact(self, K: np.ndarray, V: np.ndarray):
         B, L, N_kv = self.B, self.L, self.N_kv
@@ -295,6 +338,16 @@ class ThinKOracle:
                     self.K_T[b][l][h] = kt
                     self.K_full[b][l][h] = kr
                     self.V_all[b][l][h] = np.array(V[b, :S_b, l, h, :], dtype=F64)
+        if self.idx_v is not None:
+            # the prefix values keep their T_v channels, recent rows stay whole (same split as the keys)
+            self.V_T = [[[None] * N_kv for _ in range(L)] for _ in range(B)]
+            for b in range(B):
+                S_p = self.seq_lens[b] - self.S_recent
+                for l in range(L):
+                    for h in range(N_kv):
+                        va = self.V_all[b][l][h]
+                        self.V_T[b][l][h] = va[:S_p][:, self.idx_v[b, l, h]].copy()
+                        self.V_all[b][l][h] = va[S_p:].copy()       # from here on: the unpruned value rows only
 
     # decode, step 5
     def append(self, k_new: np.ndarray, v_new: np.ndarray):
@@ -329,6 +382,11 @@ class ThinKOracle:
                 for h in range(self.N_kv):
                     for g in range(self.G):
                         n = h * self.G + g
-                        out[b, l, n] = decode_attention(q[b, l, n], self.K_T[b][l][h], self.idx[b, l, h],
-                                                        self.K_full[b][l][h], self.V_all[b][l][h])
+                        if self.idx_v is None:
+                            out[b, l, n] = decode_attention(q[b, l, n], self.K_T[b][l][h], self.idx[b, l, h],
+                                                            self.K_full[b][l][h], self.V_all[b][l][h])
+                        else:
+                            out[b, l, n] = decode_attention_kv(q[b, l, n], self.K_T[b][l][h], self.idx[b, l, h],
+                                                               self.K_full[b][l][h], self.V_T[b][l][h],
+                                                               self.idx_v[b, l, h], self.V_all[b][l][h])
         return out

@@ -369,6 +369,70 @@ def test_value_score_against_loops():
     np.testing.assert_allclose(orc.score_value(Q, K, V), want, rtol=1e-12)
 
 
+def test_value_score_uniform_attention_closed_form():
+    # K = 0 makes every attention row uniform, so each output row is the column mean of V and the
+    # score is sqrt(rows) * |mean_j|
+    rng = np.random.default_rng(5)
+    G, S_obs, S, D = 2, 3, 11, 6
+    V = rng.normal(size=(S, D))
+    got = orc.score_value(rng.normal(size=(G, S_obs, D)), np.zeros((S, D)), V)
+    np.testing.assert_allclose(got, math.sqrt(G * S_obs) * np.abs(V.mean(axis=0)), rtol=1e-12)
+
+
+def test_value_pruning_decode_equals_zeroed_prefix_channels():
+    # ThinKV decode = ordinary ThinK decode on a value cache whose pruned channels are zero on the prefix
+    # rows (computed by the other routine); lam_v = 0 is the ThinK path itself; a channel that is zero on
+    # the prefix anyway can be pruned for free.
+    rng = np.random.default_rng(9)
+    B, L, N_q, N_kv, D, S_obs, S, R = 1, 1, 4, 2, 16, 4, 60, 8
+    K = rng.normal(size=(B, S, L, N_kv, D)) * np.exp(rng.normal(size=D))
+    V = rng.normal(size=(B, S, L, N_kv, D)) * np.exp(0.3 * rng.normal(size=D))
+    Q = rng.normal(size=(B, S_obs, L, N_q, D))
+    kv = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, R, 0.5, lam_v=0.25)
+    kv.score_select(Q, K)
+    kv.score_select_v(Q, K, V)
+    assert kv.T_v == 12 and kv.idx_v.shape == (B, L, N_kv, 12)
+    for h in range(N_kv):                      # selection = the ranked value scores of this head
+        Qg = np.stack([Q[0, :, 0, h * 2 + g] for g in range(2)])
+        s = orc.score_value(Qg, K[0, :, 0, h], V[0, :, 0, h])
+        assert set(kv.idx_v[0, 0, h]) == set(np.argsort(-s, kind="stable")[:12])
+        assert (np.diff(kv.idx_v[0, 0, h]) > 0).all()
+    kv.compact(K, V)
+    k_only = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, R, 0.5)
+    k_only.score_select(Q, K)
+    Vz = V.copy()
+    for h in range(N_kv):
+        dropped = np.setdiff1d(np.arange(D), kv.idx_v[0, 0, h])
+        Vz[0, : S - R, 0, h][:, dropped] = 0.0
+    k_only.compact(K, Vz)
+    k_new, v_new = rng.normal(size=(B, L, N_kv, D)), rng.normal(size=(B, L, N_kv, D))
+    q = rng.normal(size=(B, L, N_q, D))
+    for o in (kv, k_only):
+        o.append(k_new, v_new)
+    np.testing.assert_allclose(kv.decode_attn(q), k_only.decode_attn(q), rtol=1e-12, atol=1e-14)
+    # the tail (recent + new rows) kept its full values: the dropped channels of the output are not zero
+    assert (np.abs(kv.decode_attn(q)) > 0).all()
+    # lam_v = 0: nothing pruned
+    full = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, R, 0.5, lam_v=0.0)
+    full.score_select(Q, K)
+    full.score_select_v(Q, K, V)
+    assert (full.idx_v == np.arange(D)).all()
+    full.compact(K, V)
+    ref = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, R, 0.5)
+    ref.score_select(Q, K)
+    ref.compact(K, V)
+    for o in (full, ref):
+        o.append(k_new, v_new)
+    np.testing.assert_allclose(full.decode_attn(q), ref.decode_attn(q), rtol=1e-12, atol=1e-14)
+    # a channel that is zero on every row scores zero and is the first to go
+    V0 = V.copy()
+    V0[..., 5] = 0.0
+    z = orc.ThinKOracle(B, L, N_q, N_kv, D, [S], S_obs, R, 0.5, lam_v=1.0 / 16)
+    z.score_select(Q, K)
+    z.score_select_v(Q, K, V0)
+    assert all(5 not in z.idx_v[0, 0, h] for h in range(N_kv)) and z.T_v == 15
+
+
 # ------------------------------------------------------------------ memory model
 def test_sec31_example_13GB():
     (B, S, L, N, D, e, printed), = _rows("sec31_kv_example.txt")
