@@ -67,6 +67,7 @@ typedef struct {
   int32_t criterion;      /* thinK_criterion */
   int32_t reserved;       /* 0 */
   double lambda;          /* pruning ratio, 0 <= lambda < 1 */
+  double lambda_v;        /* pruning ratio of the value channels (App. D); 0 = values untouched (the default path) */
 } thinK_config;
 
 /* A strided view of a B x S x L x N x D tensor.  Strides are in ELEMENTS; the D
@@ -92,6 +93,9 @@ typedef struct {
    * the same number of tokens. */
   size_t model_think_bytes;
   size_t model_dense_bytes;
+  /* Only with lambda_v > 0 (else 0): */
+  size_t v_thin;    /* pruned prefix values, bf16 [rows of T_v kept channels padded to a multiple of 16] */
+  size_t perm_v;    /* uint8 [B, L, N_kv, D]: kept value channels ascending, then the pruned ones ascending */
 } thinK_sizes;
 
 typedef struct thinK_cache thinK_cache; /* opaque, host side */
@@ -120,7 +124,14 @@ const char* thinK_status_string(thinK_status s);
  *    16*step + 8*jx + r; a trailing group of 8 channels is a 256-byte block with 8 bytes per lane
  *    (pair (16*n16+2q, +1) for jx = 0,1).
  * tail_k uses the same tile layout with all D channels: [B, L, N_kv, ceil(cap/64)] tiles of D x 64,
- * cap = S_recent + max_new_tokens. */
+ * cap = S_recent + max_new_tokens.
+ * After the n_tiles(b) prompt tiles every head owns ceil(cap/64) more tiles in k_thin, which receive the
+ * tail blocks that thinK_reprune_tail thins (so the tile number above uses n_tiles(b) + ceil(cap/64)
+ * per head).
+ * v_thin (lambda_v > 0): token-major rows of Tvp = T_v rounded up to 16 bf16 elements, row t of head
+ * (b, l, h) at element v_base(b) + ((l*N_kv + h)*S_p(b) + t)*Tvp, v_base(b) = sum_{b'<b} L*N_kv*S_p(b')*Tvp;
+ * element c < T_v of a row is channel perm_v[b][l][h][c] of the value, the padding is zero.  With
+ * lambda_v > 0 the rows of tail_v are stored in the channel order perm_v[b][l][h][0..D). */
 thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens, thinK_sizes* out);
 
 /* Builds the host-side handle and writes the small device tables (lengths,
@@ -145,11 +156,33 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
 thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, int32_t layer0,
                                 int32_t nlayers, void* stream);
 
+/* Value-channel pruning (App. D, "ThinKV"), bf16 caches only.  With cfg.lambda_v > 0 the caller hands
+ * over the two extra buffers of thinK_sizes (v_thin, perm_v) right after thinK_create; the path is then
+ *   thinK_score_select_kv -> thinK_compact -> { thinK_append -> thinK_decode_attn }*
+ * (thinK_prefill takes both steps).  `scores_v` (fp64 [B, L, N_kv, D], thinK_sizes.scores bytes) may be
+ * NULL: the value scores are then not kept.  THINK_ERR_STATE if lambda_v == 0. */
+thinK_status thinK_attach_value_cache(thinK_cache* c, void* v_thin, void* perm_v, void* scores_v);
+
+/* thinK_score_select plus the value-channel score of App. D, Eqs. 3-4:
+ *   Score_v[j] = || softmax(Q[-S_obs:] K^T / sqrt(D)) V[:, j] ||_F,   I_v = Top_T(Score_v, T_v),
+ * T_v = floor((1 - lambda_v) D).  All S_b rows of K and V enter, no causal mask inside the window
+ * (the formula has none), the G query heads of a group are stacked row-wise as for the key score, ties
+ * go to the lower channel.  Both products run on tensor cores in bf16 with fp32 accumulation, the
+ * softmax weights as a bf16 pair hi + lo; column norms in fp64.  Against an fp64 evaluation the scores
+ * carry a relative error of about 1e-5, so two channels whose scores are closer than that may swap.
+ * Writes perm_v (kept channels ascending, then the rest ascending).  `v` as for thinK_compact. */
+thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v,
+                                   int32_t layer0, int32_t nlayers, void* stream);
+
 /* Prefill, Sec. 3.3: builds the two-part key cache for the given layers from
  * the idx thinK_score_select stored: K_T[t][c] = K[t][idx[c]] for t < S_p, and
  * the last S_recent rows of K and V copied unpruned to the tail.  After this
  * call K may be released by the caller; V rows [0, S_p) of `v` stay BORROWED:
- * thinK_decode_attn reads them in place on every step. */
+ * thinK_decode_attn reads them in place on every step.
+ * With lambda_v > 0 (after thinK_score_select_kv) the prefix values are thinned too:
+ * V_T[t][c] = V[t][perm_v[c]], c < T_v, written to v_thin; the recent rows keep all D channels
+ * (declared reading: App. D gives the criterion only; the split mirrors the keys').  `v` is then
+ * not borrowed. */
 thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0, int32_t nlayers,
                            void* stream);
 
@@ -197,7 +230,9 @@ thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, 
  * the weighted sum of all value rows (prompt V in place + tail).
  *   q, out: dense [B, nlayers, N_q, D] in the cache dtype.
  * bf16: fp32 accumulation; fp32: logits in fp64, fp32 accumulation of p.V.
- * All layers in the range must hold the same number of tail tokens. */
+ * All layers in the range must hold the same number of tail tokens.
+ * With lambda_v > 0 a pruned value channel of a prefix token counts as zero: output channel j sums the
+ * tail tokens' share always and the prefix tokens' share only if j is kept. */
 thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
                                void* stream);
 

@@ -33,7 +33,7 @@ class Config(C.Structure):
     _fields_ = [("B", C.c_int32), ("L", C.c_int32), ("N_q", C.c_int32), ("N_kv", C.c_int32), ("D", C.c_int32),
                 ("S_max", C.c_int32), ("S_obs", C.c_int32), ("S_recent", C.c_int32),
                 ("max_new_tokens", C.c_int32), ("dtype", C.c_int32), ("criterion", C.c_int32),
-                ("reserved", C.c_int32), ("lam", C.c_double)]
+                ("reserved", C.c_int32), ("lam", C.c_double), ("lam_v", C.c_double)]
 
 
 class Tensor5(C.Structure):
@@ -44,7 +44,7 @@ class Tensor5(C.Structure):
 class Sizes(C.Structure):
     _fields_ = [("k_thin", C.c_size_t), ("tail_k", C.c_size_t), ("tail_v", C.c_size_t), ("idx", C.c_size_t),
                 ("scores", C.c_size_t), ("workspace", C.c_size_t), ("model_think_bytes", C.c_size_t),
-                ("model_dense_bytes", C.c_size_t)]
+                ("model_dense_bytes", C.c_size_t), ("v_thin", C.c_size_t), ("perm_v", C.c_size_t)]
 
 
 EXPORTS = {
@@ -55,6 +55,8 @@ EXPORTS = {
     "thinK_score_select": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_compact": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_prefill": (C.c_int, [C.c_void_p, Tensor5, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_attach_value_cache": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
+    "thinK_score_select_kv": (C.c_int, [C.c_void_p, Tensor5, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_prefill_evicted": (C.c_int, [C.c_void_p, Tensor5, Tensor5, Tensor5, C.c_void_p, C.c_int64, C.c_int32,
                                         C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_v_kept_bytes": (C.c_size_t, [C.c_void_p]),
@@ -105,9 +107,10 @@ def tensor5(t: Optional[torch.Tensor]) -> Tensor5:
     return Tensor5(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2), t.stride(3))
 
 
-def make_config(B, L, N_q, N_kv, D, S_max, S_obs, S_recent, max_new_tokens, lam, dtype, criterion=SCORE_QUERY_DRIVEN):
+def make_config(B, L, N_q, N_kv, D, S_max, S_obs, S_recent, max_new_tokens, lam, dtype, criterion=SCORE_QUERY_DRIVEN,
+                lam_v=0.0):
     return Config(B, L, N_q, N_kv, D, S_max, S_obs, S_recent, max_new_tokens,
-                  dtype if isinstance(dtype, int) else _dtype_code(dtype), criterion, 0, float(lam))
+                  dtype if isinstance(dtype, int) else _dtype_code(dtype), criterion, 0, float(lam), float(lam_v))
 
 
 def thinK_cache_bytes(cfg: Config, seq_lens: Sequence[int]) -> Sizes:
@@ -162,6 +165,29 @@ class ThinKCache:
                                     self.scores.data_ptr() if self.scores is not None else None,
                                     self.workspace.data_ptr(), C.byref(h)), "thinK_create")
         self.handle = h
+        self.T_v = thinK_T(cfg.lam_v, cfg.D)
+        self.v_thin = self.perm_v = None
+        if cfg.lam_v > 0:                      # value-channel pruning: two more caller-owned buffers
+            self.v_thin, self.perm_v = mk(self.sizes.v_thin), mk(self.sizes.perm_v)
+            self.scores_v = mk(self.sizes.scores) if keep_scores else None
+            _check(lib.thinK_attach_value_cache(self.handle, self.v_thin.data_ptr(), self.perm_v.data_ptr(),
+                                                self.scores_v.data_ptr() if self.scores_v is not None else None),
+                   "thinK_attach_value_cache")
+
+    def score_select_kv(self, q_obs: torch.Tensor, k: torch.Tensor, v: torch.Tensor, layer0=0, nlayers=None, stream=None):
+        """Key scores + value scores (App. D) and both selections."""
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        _check(lib.thinK_score_select_kv(self.handle, tensor5(q_obs), tensor5(k), tensor5(v), layer0, nlayers,
+                                         _stream_ptr(stream)), "thinK_score_select_kv")
+
+    def scores_v_tensor(self) -> torch.Tensor:
+        c = self.cfg
+        return self.scores_v[: c.B * c.L * c.N_kv * c.D * 8].view(torch.float64).view(c.B, c.L, c.N_kv, c.D)
+
+    def perm_v_tensor(self) -> torch.Tensor:
+        """uint8 [B, L, N_kv, D]: kept value channels ascending ([..., :T_v]), then the pruned ones."""
+        c = self.cfg
+        return self.perm_v[: c.B * c.L * c.N_kv * c.D].view(c.B, c.L, c.N_kv, c.D)
 
     # -- the four calls of the path -------------------------------------
     def score_select(self, q_obs: Optional[torch.Tensor], k: torch.Tensor, layer0=0, nlayers=None, stream=None):
@@ -327,4 +353,21 @@ def tail_logical(cache: ThinKCache, b: int, l: int, h: int):
     m = cache.repruned_len(l)                              # these tokens now live in k_thin
     keys = unpack_tiles(flat[unit * ttc * per:(unit + 1) * ttc * per], ttc, c.D, n)[m:]
     vals = cache.tail_v.view(cache.torch_dtype)[unit * cap * c.D:(unit * cap + n) * c.D].view(n, c.D)[m:]
+    if cache.perm_v is not None:                           # stored in the permuted channel order: undo it
+        perm = cache.perm_v_tensor()[b, l, h].long()
+        out = torch.empty_like(vals)
+        out[:, perm] = vals
+        vals = out
     return keys, vals
+
+
+def v_thin_logical(cache: ThinKCache, b: int, l: int, h: int) -> torch.Tensor:
+    """Thinned prefix values of one head, [S_p, T_v] (kept channels ascending)."""
+    c = cache.cfg
+    Tvp = (cache.T_v + 15) // 16 * 16
+    base = sum(c.L * c.N_kv * (cache.seq_lens[bb] - c.S_recent) * Tvp for bb in range(b))
+    S_p = cache.seq_lens[b] - c.S_recent
+    off = base + (l * c.N_kv + h) * S_p * Tvp
+    rows = cache.v_thin.view(cache.torch_dtype)[off: off + S_p * Tvp].view(S_p, Tvp)
+    assert (rows[:, cache.T_v:] == 0).all(), "padding channels of v_thin must be zero"
+    return rows[:, : cache.T_v]

@@ -194,7 +194,15 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
     const Tin* ks = (const Tin*)p.k.ptr + b * p.k.sb + srow * p.k.ss + (int64_t)sl * p.k.sl + (int64_t)h * p.k.sn + ck * CH;
     const Tin* vs = (const Tin*)p.v.ptr + b * p.v.sb + srow * p.v.ss + (int64_t)sl * p.v.sl + (int64_t)h * p.v.sn + ck * CH;
     uint4 kv = __ldg((const uint4*)ks);
-    uint4 vv = __ldg((const uint4*)vs);
+    uint4 vv;
+    if (p.perm_v) {                                 // channel c of the stored row = channel perm_v[c] of the source
+      const uint8_t* pm = p.perm_v + unit * p.D + ck * CH;
+      Tin* e = (Tin*)&vv;
+#pragma unroll
+      for (int j = 0; j < CH; ++j) e[j] = vs[(int)pm[j] - ck * CH];
+    } else {
+      vv = __ldg((const uint4*)vs);
+    }
     const int u = p.pos0 + r;                       // position in the tail
     *(uint4*)((Tin*)p.tail_v + (unit * p.cap + u) * p.D + ck * CH) = vv;
     unsigned char* tile = (unsigned char*)p.tail_k + (unit * p.tail_tiles_cap + u / kTileTokens) * (int64_t)p.D * kTileTokens * E;
@@ -206,6 +214,35 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
       if (E == 2) *(Tin*)(tile + frag_elem_byte(p.D, c, uu)) = kk[j];
       else *(Tin*)(tile + c * kTileTokens * E + tile_swz_bytes(c, uu, E)) = kk[j];
     }
+  }
+}
+
+// Value-channel pruning (paper App. D): V_T[t][c] = V[t][perm_v[c]] for c < T_v, rows of Tvp elements
+// (zero padded), t < S_p.  One thread builds one 16-byte piece of one thinned row.
+__global__ void __launch_bounds__(256) k_compact_value(const CompactValueParams p) {
+  const int cpr = p.Tvp / 8;
+  const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.S_pmax * cpr;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int ck = i % cpr;
+    int64_t r1 = i / cpr;
+    const int t = r1 % p.S_pmax; r1 /= p.S_pmax;
+    const int h = r1 % p.N_kv; r1 /= p.N_kv;
+    const int l = p.layer0 + (int)(r1 % p.nlayers);
+    const int b = (int)(r1 / p.nlayers);
+    const int S_p = p.seq_len[b] - p.R;
+    if (t >= S_p) continue;
+    const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+    const uint16_t* src = (const uint16_t*)p.v.ptr + b * p.v.sb + (int64_t)t * p.v.ss + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;
+    const uint8_t* pm = p.perm_v + unit * p.D + ck * 8;
+    uint32_t w[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c = ck * 8 + 2 * j;
+      const uint32_t lo = c < p.Tv ? src[pm[2 * j]] : 0u, hi = c + 1 < p.Tv ? src[pm[2 * j + 1]] : 0u;
+      w[j] = lo | (hi << 16);
+    }
+    uint16_t* dst = (uint16_t*)p.v_thin + p.v_thin_base[b] + ((int64_t)(l * p.N_kv + h) * S_p + t) * p.Tvp + ck * 8;
+    *(uint4*)dst = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
@@ -231,6 +268,14 @@ __global__ void __launch_bounds__(256) k_gather_rows(const GatherRowsParams p) {
 }
 
 }  // namespace
+
+cudaError_t launch_compact_value(const CompactValueParams& p, cudaStream_t s) {
+  const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.S_pmax * (p.Tvp / 8);
+  if (total <= 0) return cudaSuccess;
+  const int64_t want = (total + 255) / 256;
+  k_compact_value<<<(int)(want < (int64_t)kSMs * 32 ? want : (int64_t)kSMs * 32), 256, 0, s>>>(p);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_gather_rows(const GatherRowsParams& p, int dtype, cudaStream_t s) {
   const int E = dtype == THINK_BF16 ? 2 : 4;

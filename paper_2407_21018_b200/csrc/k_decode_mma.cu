@@ -96,7 +96,9 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-template <int D, int G>
+// VT: the prefix values are thinned as well (App. D); everything about values then lives in the
+// permuted channel order and the output is un-permuted when it is written.
+template <int D, int G, bool VT>
 __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParams p) {
   static_assert(D == 64 || D == 128, "head dimension");
   constexpr int NT = D / 8;              // n-tiles of the output
@@ -142,6 +144,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
   // full across unit boundaries; the consumer below follows the same sequence.
   long long pf = f0;                                  // first tile not yet handed to the producer
   int islot = 0, i_left = 0, i_kstep = 0;
+  int i_vck = CPR;                                    // 16-byte chunks per value row of the region
   long long i_vrow = 0;
   const unsigned char* ikl = nullptr;
   const unsigned char* iv = nullptr;
@@ -168,10 +171,17 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       const int je = j1 < nthin ? j1 : nthin;
       ntiles = je - j0;
       i_kstep = Tp * 32;
-      i_vrow = p.v.ss * 2;
       k0 = (const unsigned char*)p.k_thin + (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (nthin + p.re_cap) + j0) * (int64_t)Tp * 128;
-      v0 = (const unsigned char*)((const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn) +
-           (int64_t)j0 * kTileTokens * i_vrow;
+      if (VT) {
+        i_vrow = p.Tvp * 2;
+        i_vck = p.Tvp >> 3;
+        v0 = (const unsigned char*)p.v_thin +
+             (p.v_thin_base[b] + ((int64_t)(l * p.N_kv + h) * (p.seq_len[b] - p.R) + (int64_t)j0 * kTileTokens) * p.Tvp) * 2;
+      } else {
+        i_vrow = p.v.ss * 2;
+        v0 = (const unsigned char*)((const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn) +
+             (int64_t)j0 * kTileTokens * i_vrow;
+      }
       i_left = min(p.seq_len[b] - p.R, je * kTileTokens) - j0 * kTileTokens;
     } else if (j0 - nthin < p.n_re) {
       // tail blocks that were re-pruned: keys thinned like the prefix, values still in the tail buffer
@@ -179,6 +189,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       ntiles = je - jb;
       i_kstep = Tp * 32;
       i_vrow = D * 2;
+      if (VT) i_vck = CPR;
       k0 = (const unsigned char*)p.k_thin +
            (p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (nthin + p.re_cap) + nthin + jb) * (int64_t)Tp * 128;
       v0 = (const unsigned char*)p.tail_v + (unit_abs * p.cap + (int64_t)jb * kTileTokens) * D * 2;
@@ -188,6 +199,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       ntiles = je - jb;
       i_kstep = D * 32;
       i_vrow = D * 2;
+      if (VT) i_vck = CPR;
       k0 = (const unsigned char*)p.tail_k + (unit_abs * p.tail_tiles_cap + jb) * (int64_t)D * 128;
       v0 = (const unsigned char*)p.tail_v + (unit_abs * p.cap + (int64_t)jb * kTileTokens) * D * 2;
       i_left = min(p.n_tail, je * kTileTokens) - jb * kTileTokens;
@@ -209,18 +221,20 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       if (lane * 16 < krem) cp_async16(kd + nfull * 512, ikl + nfull * 512);
       const unsigned char* vs = iv;
       const long long rstep = RPI * i_vrow;
-      if (i_left >= kStepTokens) {
+      if (!VT || vlane_ck < i_vck) {                  // thinned rows are shorter: the other lanes sit out
+        if (i_left >= kStepTokens) {
 #pragma unroll
-        for (int it = 0; it < VIT; ++it) {
-          cp_async16(sb + kKSlot + vdst_off[it], vs);
-          vs += rstep;
-        }
-      } else {                                        // last step of a region: zero-fill missing rows
+          for (int it = 0; it < VIT; ++it) {
+            cp_async16(sb + kKSlot + vdst_off[it], vs);
+            vs += rstep;
+          }
+        } else {                                      // last step of a region: zero-fill missing rows
 #pragma unroll
-        for (int it = 0; it < VIT; ++it) {
-          const bool ok = it * RPI + vlane_row < i_left;
-          cp_async16_zfill(sb + kKSlot + vdst_off[it], ok ? vs : i_vsafe, ok ? 16 : 0);
-          vs += rstep;
+          for (int it = 0; it < VIT; ++it) {
+            const bool ok = it * RPI + vlane_row < i_left;
+            cp_async16_zfill(sb + kKSlot + vdst_off[it], ok ? vs : i_vsafe, ok ? 16 : 0);
+            vs += rstep;
+          }
         }
       }
       i_left -= kStepTokens;
@@ -314,6 +328,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       if (q_kind != (int)thin) { load_q(thin); q_kind = thin; }
       const int n16 = thin ? n16_thin : KS;
       const bool has8 = thin && has8_thin;
+      const int npv = (VT && cr == 0) ? (p.Tvp >> 4) : NT / 2;   // pairs of n-tiles the region's values fill
       for (int left = ntok; left > 0; left -= kStepTokens) {
         cp_wait<kStages - 2>();
         __syncwarp();       // this step's data has landed; every lane is done with the previous slot
@@ -373,6 +388,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
         // O += P . V : value rows through ldmatrix.trans (tokens become the contraction index)
 #pragma unroll
         for (int np = 0; np < NT / 2; ++np) {
+          if (VT && np >= npv) continue;
           uint32_t v0, v1, v2, v3;
           ldmatrix_x4_trans(vbase + vld_off[np], v0, v1, v2, v3);
           mma16816(o[2 * np], pa0, pa2, v0, v1);
@@ -386,12 +402,19 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
     lsum += __shfl_xor_sync(0xffffffffu, lsum, 2);
     const bool complete = (f == ustart) && (seg_end == uend);
     __nv_bfloat16* outp = (__nv_bfloat16*)p.out + ((int64_t)(b * p.nlayers + ll) * p.N_q + h * G) * D;
+    const uint8_t* perm = VT ? p.perm_v + unit_abs * D : nullptr;   // accumulator column c is output channel perm[c]
     if (complete) {
       if (row < G) {
         const float inv = 1.f / lsum;
 #pragma unroll
-        for (int t = 0; t < NT; ++t)
-          *(uint32_t*)(outp + row * D + 8 * t + 2 * qd) = pack_bf16(o[t][0] * inv, o[t][1] * inv);
+        for (int t = 0; t < NT; ++t) {
+          if (VT) {
+            outp[row * D + perm[8 * t + 2 * qd]] = __float2bfloat16_rn(o[t][0] * inv);
+            outp[row * D + perm[8 * t + 2 * qd + 1]] = __float2bfloat16_rn(o[t][1] * inv);
+          } else {
+            *(uint32_t*)(outp + row * D + 8 * t + 2 * qd) = pack_bf16(o[t][0] * inv, o[t][1] * inv);
+          }
+        }
       }
     } else {
       uint8_t* rec = p.records + ((size_t)wk * 2 + (f == f0 ? 0 : 1)) * rec_bytes;
@@ -437,8 +460,11 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
           for (int k = 0; k < EPL; ++k) acc[k] = fmaf(ov[k], __shfl_sync(0xffffffffu, w, (lane + 32 * k) / D), acc[k]);
         }
 #pragma unroll
-        for (int k = 0; k < EPL; ++k)
-          outp[lane + 32 * k] = __float2bfloat16_rn(acc[k] / __shfl_sync(0xffffffffu, Lsum, (lane + 32 * k) / D));
+        for (int k = 0; k < EPL; ++k) {
+          const int i = lane + 32 * k;
+          const int oi = VT ? (i / D) * D + perm[i % D] : i;
+          outp[oi] = __float2bfloat16_rn(acc[k] / __shfl_sync(0xffffffffu, Lsum, i / D));
+        }
         __syncwarp();
         if (lane == 0) p.counters[unit_call] = 0u;
       }
@@ -450,12 +476,15 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
 
 template <int D, int G>
 cudaError_t launch_mma(const DecodeParams& p, cudaStream_t s) {
-  k_decode_mma<D, G><<<p.grid, kWarps * 32, kSmemBytes, s>>>(p);
+  if (p.v_thin) k_decode_mma<D, G, true><<<p.grid, kWarps * 32, kSmemBytes, s>>>(p);
+  else k_decode_mma<D, G, false><<<p.grid, kWarps * 32, kSmemBytes, s>>>(p);
   return cudaGetLastError();
 }
 template <int D, int G>
 cudaError_t setup_mma() {
-  return cudaFuncSetAttribute(k_decode_mma<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(k_decode_mma<D, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_decode_mma<D, G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
 }
 
 #define THINK_MMA_DISPATCH(FN, ...)                                   \

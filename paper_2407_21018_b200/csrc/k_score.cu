@@ -41,28 +41,6 @@ __device__ __forceinline__ uint4 ldg16(const void* p) {
   return v;
 }
 
-// Rank-count selection of one head by one warp: channel j is kept when fewer than T channels
-// beat it, where k beats j if s[k] > s[j] or (s[k] == s[j] and k < j).  Output ascending.
-__device__ void select_head(const double* s, int D, int T, uint8_t* out, int lane) {
-  int base = 0;
-  for (int j0 = 0; j0 < D; j0 += 32) {
-    int j = j0 + lane;
-    bool keep = false;
-    if (j < D) {
-      double sj = s[j];
-      int rank = 0;
-      for (int k = 0; k < D; ++k) {
-        double sk = s[k];
-        rank += (sk > sj) || (sk == sj && k < j);
-      }
-      keep = rank < T;
-    }
-    unsigned m = __ballot_sync(0xffffffffu, keep);
-    if (keep) out[base + __popc(m & ((1u << lane) - 1u))] = (uint8_t)j;
-    base += __popc(m);
-  }
-}
-
 template <typename Tin, bool L1, bool TOK>
 __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const ScoreParams p) {
   constexpr int CH = Chunk<Tin>::CH;
@@ -216,7 +194,7 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
   const int warp = tid >> 5, lane = tid & 31;
   for (int hh = warp; hh < heads; hh += kScoreThreads / 32) {
     const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h_first + hh;
-    select_head(red + hh * p.D, p.D, p.T, p.idx + unit * p.T, lane);
+    select_head(red + hh * p.D, p.D, p.T, p.idx + unit * p.T, lane, false);
     if (p.scores)
       for (int j = lane; j < p.D; j += 32) p.scores[unit * p.D + j] = red[hh * p.D + j];
   }

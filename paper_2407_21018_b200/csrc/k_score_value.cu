@@ -1,0 +1,284 @@
+// Value-channel scores and their top-T_v (paper App. D, Eqs. 3-4), bf16:
+//   Score_v[j] = || softmax(Q[-S_obs:] K^T / sqrt(D)) V[:, j] ||_F ,  I_v = Top_T(Score_v, T_v).
+//
+// Unlike the key score this has no closed form: it is the attention output of the window's queries
+// (the G query heads of the group stacked: M = G * S_obs rows) over the whole prompt, i.e. two dense
+// contractions per head, so it runs on tensor cores (mma.sync m16n8k16, bf16 in, fp32 accumulate).
+//  * A CTA owns (token split, block of up to 128 query rows, unit (b, l, h)); warp w owns 16 rows.
+//    K and V tiles of 64 tokens are staged with cp.async into a two-stage ring shared by the warps
+//    (rows XOR-swizzled by 16-byte chunk so that ldmatrix is conflict-free).
+//  * Online softmax per row in the exp2 domain.  The weights enter the second product as a bf16
+//    pair hi + lo (two MMAs), so their rounding error is 2^-17 instead of 2^-9: the scores then agree
+//    with an fp64 evaluation to ~1e-5 and the ranking is stable against it.
+//  * Every CTA leaves (m, l, O) of its rows in the workspace; the CTA that takes the unit's last
+//    ticket merges the splits in order, forms the column norms in fp64 and ranks the channels.
+#include <math.h>
+
+#include "think_internal.h"
+
+namespace think {
+namespace {
+
+constexpr int kVTile = 64;        // tokens per staged tile
+constexpr int kVStages = 2;
+constexpr int kRowGroups = 8;     // row groups of the finaliser's column sums
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, int src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+// (lo, hi) -> packed bf16 pair of the values and of what the rounding left over
+__device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& hi, uint32_t& lo, float& sum) {
+  const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1);
+  const float r0 = x0 - __bfloat162float(h0), r1 = x1 - __bfloat162float(h1);
+  const __nv_bfloat16 l0 = __float2bfloat16_rn(r0), l1 = __float2bfloat16_rn(r1);
+  hi = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+  lo = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+  sum += (__bfloat162float(h0) + __bfloat162float(l0)) + (__bfloat162float(h1) + __bfloat162float(l1));
+}
+
+template <int D>
+__global__ void __launch_bounds__(256, 1) k_score_value(const ValueScoreParams p) {
+  constexpr int KS = D / 16, NT = D / 8;
+  constexpr int CPR = D * 2 / 16;            // 16-byte chunks per row
+  constexpr int ROWB = D * 2;
+  constexpr int kTileBytes = kVTile * ROWB;
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ int s_last;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x;
+  const int qd = lane & 3, frow = lane >> 2;
+  const int split = blockIdx.x, rb = blockIdx.y, ucall = blockIdx.z;
+  const int h = ucall % p.N_kv, bl = ucall / p.N_kv;
+  const int ll = bl % p.nlayers, b = bl / p.nlayers, l = p.layer0 + ll;
+  const int S_b = p.seq_len[b];
+  const int ntile_all = (S_b + kVTile - 1) / kVTile;
+  const int per = (ntile_all + p.nsplit - 1) / p.nsplit;
+  const int t0 = min(S_b, split * per * kVTile), t1 = min(S_b, (split + 1) * per * kVTile);
+  const int ntl = (t1 - t0 + kVTile - 1) / kVTile;
+
+  // ---- query rows of this warp (A operand).  Row r of the unit = query head h*G + r / S_obs, window row r % S_obs.
+  const int rA = rb * p.MB + warp * 16 + frow, rB = rA + 8;
+  uint32_t qa[KS][4];
+  {
+    const __nv_bfloat16* qbase = (const __nv_bfloat16*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl;
+    const bool okA = rA < p.M, okB = rB < p.M;
+    const __nv_bfloat16* qA = qbase + (int64_t)(okA ? rA % p.S_obs : 0) * p.q.ss + (int64_t)(h * p.G + (okA ? rA / p.S_obs : 0)) * p.q.sn;
+    const __nv_bfloat16* qB = qbase + (int64_t)(okB ? rB % p.S_obs : 0) * p.q.ss + (int64_t)(h * p.G + (okB ? rB / p.S_obs : 0)) * p.q.sn;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const int c = 16 * ks + 2 * qd;
+      qa[ks][0] = okA ? *(const uint32_t*)(qA + c) : 0u;
+      qa[ks][1] = okB ? *(const uint32_t*)(qB + c) : 0u;
+      qa[ks][2] = okA ? *(const uint32_t*)(qA + c + 8) : 0u;
+      qa[ks][3] = okB ? *(const uint32_t*)(qB + c + 8) : 0u;
+    }
+  }
+
+  const __nv_bfloat16* kg = (const __nv_bfloat16*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn;
+  const __nv_bfloat16* vg = (const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;
+  const uint32_t sbase = smem_u32(smem);
+  auto load_tile = [&](int stage, int tok0) {
+    const uint32_t kd = sbase + stage * 2 * kTileBytes, vd = kd + kTileBytes;
+    for (int i = tid; i < kVTile * CPR; i += nthreads) {
+      const int r = i / CPR, ck = i % CPR;
+      const bool ok = tok0 + r < t1;                 // rows past the range are zero-filled
+      const int64_t t = ok ? tok0 + r : t0;
+      const uint32_t off = r * ROWB + ((ck ^ (r & 7)) << 4);
+      cp_async16_zfill(kd + off, kg + t * p.k.ss + ck * 8, ok ? 16 : 0);
+      cp_async16_zfill(vd + off, vg + t * p.v.ss + ck * 8, ok ? 16 : 0);
+    }
+  };
+
+  // ---- per-lane ldmatrix offsets inside a tile
+  const int mi = lane >> 3;
+  // keys (not transposed): matrix mi = (token block mi>>1, channel half mi&1) of a pair of token blocks
+  const int k_row = ((mi >> 1) << 3) + (lane & 7);
+  // values (transposed): matrix mi = (token half mi&1, n-tile mi>>1) of a pair of n-tiles
+  const int v_row = ((mi & 1) << 3) + (lane & 7);
+
+  const float scale = 1.4426950408889634f / sqrtf((float)D);
+  float mA = -INFINITY, mB = -INFINITY, lA = 0.f, lB = 0.f;
+  float o[NT][4];
+#pragma unroll
+  for (int t = 0; t < NT; ++t) o[t][0] = o[t][1] = o[t][2] = o[t][3] = 0.f;
+
+  if (ntl > 0) load_tile(0, t0);
+  cp_commit();
+  for (int it = 0; it < ntl; ++it) {
+    if (it + 1 < ntl) load_tile((it + 1) & 1, t0 + (it + 1) * kVTile);
+    cp_commit();
+    cp_wait<1>();
+    __syncthreads();
+    const uint32_t kt = sbase + (it & 1) * 2 * kTileBytes, vt = kt + kTileBytes;
+    const int nvalid = min(kVTile, t1 - (t0 + it * kVTile));
+    // S = Q K^T for the 64 tokens of the tile
+    float s[8][4];
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) s[nb][0] = s[nb][1] = s[nb][2] = s[nb][3] = 0.f;
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+#pragma unroll
+      for (int nbp = 0; nbp < 4; ++nbp) {
+        const int r = 16 * nbp + k_row, ck = 2 * ks + (mi & 1);
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4(kt + r * ROWB + ((ck ^ (r & 7)) << 4), b0, b1, b2, b3);
+        mma16816(s[2 * nbp], qa[ks], b0, b1);
+        mma16816(s[2 * nbp + 1], qa[ks], b2, b3);
+      }
+    }
+    // logits in the exp2 domain, masked past the range; row maxima
+    float mxA = -INFINITY, mxB = -INFINITY;
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) {
+      const int c = 8 * nb + 2 * qd;
+      s[nb][0] = c < nvalid ? s[nb][0] * scale : -INFINITY;
+      s[nb][1] = c + 1 < nvalid ? s[nb][1] * scale : -INFINITY;
+      s[nb][2] = c < nvalid ? s[nb][2] * scale : -INFINITY;
+      s[nb][3] = c + 1 < nvalid ? s[nb][3] * scale : -INFINITY;
+      mxA = fmaxf(mxA, fmaxf(s[nb][0], s[nb][1]));
+      mxB = fmaxf(mxB, fmaxf(s[nb][2], s[nb][3]));
+    }
+    mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 1));
+    mxA = fmaxf(mxA, __shfl_xor_sync(0xffffffffu, mxA, 2));
+    mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 1));
+    mxB = fmaxf(mxB, __shfl_xor_sync(0xffffffffu, mxB, 2));
+    const float nA = fmaxf(mA, mxA), nB = fmaxf(mB, mxB);     // finite: a tile holds at least one token
+    const float cA = ex2(mA - nA), cB = ex2(mB - nB);
+    mA = nA; mB = nB;
+    lA *= cA; lB *= cB;
+#pragma unroll
+    for (int t = 0; t < NT; ++t) { o[t][0] *= cA; o[t][1] *= cA; o[t][2] *= cB; o[t][3] *= cB; }
+    // O += P V, 16 tokens at a time; P as hi + lo
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      uint32_t ahi[4], alo[4];
+      split_pair(ex2(s[2 * j][0] - mA), ex2(s[2 * j][1] - mA), ahi[0], alo[0], lA);
+      split_pair(ex2(s[2 * j][2] - mB), ex2(s[2 * j][3] - mB), ahi[1], alo[1], lB);
+      split_pair(ex2(s[2 * j + 1][0] - mA), ex2(s[2 * j + 1][1] - mA), ahi[2], alo[2], lA);
+      split_pair(ex2(s[2 * j + 1][2] - mB), ex2(s[2 * j + 1][3] - mB), ahi[3], alo[3], lB);
+#pragma unroll
+      for (int np = 0; np < NT / 2; ++np) {
+        const int r = 16 * j + v_row, ck = 2 * np + (mi >> 1);
+        uint32_t v0, v1, v2, v3;
+        ldmatrix_x4_trans(vt + r * ROWB + ((ck ^ (r & 7)) << 4), v0, v1, v2, v3);
+        mma16816(o[2 * np], ahi, v0, v1);
+        mma16816(o[2 * np], alo, v0, v1);
+        mma16816(o[2 * np + 1], ahi, v2, v3);
+        mma16816(o[2 * np + 1], alo, v2, v3);
+      }
+    }
+    __syncthreads();      // everyone is done with this stage before it is refilled
+  }
+  cp_wait<0>();
+
+  // ---- partial state of this CTA's rows
+  lA += __shfl_xor_sync(0xffffffffu, lA, 1);
+  lA += __shfl_xor_sync(0xffffffffu, lA, 2);
+  lB += __shfl_xor_sync(0xffffffffu, lB, 1);
+  lB += __shfl_xor_sync(0xffffffffu, lB, 2);
+  const size_t rec_floats = (size_t)p.MB * (2 + D);
+  {
+    float* rec = p.partials + ((size_t)(ucall * p.nrb + rb) * p.nsplit + split) * rec_floats;
+    const int la = warp * 16 + frow, lb = la + 8;
+    if (qd == 0) { rec[la] = mA; rec[lb] = mB; rec[p.MB + la] = lA; rec[p.MB + lb] = lB; }
+    float* oa = rec + 2 * p.MB + (size_t)la * D + 2 * qd;
+    float* ob = rec + 2 * p.MB + (size_t)lb * D + 2 * qd;
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+      *(float2*)(oa + 8 * t) = make_float2(o[t][0], o[t][1]);
+      *(float2*)(ob + 8 * t) = make_float2(o[t][2], o[t][3]);
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(p.counters + ucall, 1u) == (uint32_t)(p.nrb * p.nsplit - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  // ---- finaliser: merge the splits row by row, column norms over all M rows, ranking
+  float* w = (float*)smem;                                   // [nsplit][M]: weight of a split's row / its denominator
+  double* en = (double*)(smem + (((size_t)p.nsplit * p.M * 4 + 15) & ~(size_t)15));   // [kRowGroups][D]
+  double* sc = en + kRowGroups * D;                          // [D]
+  const float* ubase = p.partials + (size_t)ucall * p.nrb * p.nsplit * rec_floats;
+  for (int r = tid; r < p.M; r += nthreads) {
+    const float* rrec = ubase + (size_t)(r / p.MB) * p.nsplit * rec_floats;
+    const int rl = r % p.MB;
+    float mx = -INFINITY;
+    for (int sp = 0; sp < p.nsplit; ++sp) mx = fmaxf(mx, __ldcg(rrec + sp * rec_floats + rl));
+    float den = 0.f;
+    for (int sp = 0; sp < p.nsplit; ++sp)
+      den += __ldcg(rrec + sp * rec_floats + p.MB + rl) * exp2f(__ldcg(rrec + sp * rec_floats + rl) - mx);
+    for (int sp = 0; sp < p.nsplit; ++sp) w[sp * p.M + r] = exp2f(__ldcg(rrec + sp * rec_floats + rl) - mx) / den;
+  }
+  __syncthreads();
+  for (int item = tid; item < kRowGroups * D; item += nthreads) {
+    const int rg = item / D, j = item % D;
+    double e = 0.0;
+    for (int r = rg; r < p.M; r += kRowGroups) {
+      const float* rrec = ubase + (size_t)(r / p.MB) * p.nsplit * rec_floats + 2 * p.MB + (size_t)(r % p.MB) * D + j;
+      float x = 0.f;
+      for (int sp = 0; sp < p.nsplit; ++sp) x = fmaf(__ldcg(rrec + sp * rec_floats), w[sp * p.M + r], x);
+      e = fma((double)x, (double)x, e);
+    }
+    en[rg * D + j] = e;
+  }
+  __syncthreads();
+  for (int j = tid; j < D; j += nthreads) {
+    double e = 0.0;
+    for (int rg = 0; rg < kRowGroups; ++rg) e += en[rg * D + j];
+    sc[j] = sqrt(e);
+  }
+  __syncthreads();
+  const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+  if (warp == 0) {
+    select_head(sc, D, p.Tv, p.perm_v + unit * D, lane, true);
+    if (p.scores_v)
+      for (int j = lane; j < D; j += 32) p.scores_v[unit * D + j] = sc[j];
+  }
+  if (tid == 0) p.counters[ucall] = 0u;   // ready for the next launch
+}
+
+constexpr int smem_bytes(int D) { return kVStages * 2 * kVTile * D * 2; }
+
+}  // namespace
+
+size_t score_value_record_bytes(int MB, int D) { return (size_t)MB * (2 + D) * sizeof(float); }
+
+cudaError_t score_value_setup(int D) {
+  if (D == 128) return cudaFuncSetAttribute(k_score_value<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128));
+  if (D == 64) return cudaFuncSetAttribute(k_score_value<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64));
+  return cudaErrorInvalidValue;
+}
+
+// threads = 32 * (MB / 16): one warp per 16 query rows of the row block
+cudaError_t launch_score_value(const ValueScoreParams& p, int threads, cudaStream_t s) {
+  dim3 grid(p.nsplit, p.nrb, p.B * p.nlayers * p.N_kv);
+  if (p.D == 128) k_score_value<128><<<grid, threads, smem_bytes(128), s>>>(p);
+  else if (p.D == 64) k_score_value<64><<<grid, threads, smem_bytes(64), s>>>(p);
+  else return cudaErrorInvalidValue;
+  return cudaGetLastError();
+}
+
+}  // namespace think

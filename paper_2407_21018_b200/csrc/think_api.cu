@@ -15,14 +15,22 @@ namespace {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // byte offsets inside the workspace
-  size_t seq_len, cum_thin, thin_tile_base, error, score_counters, decode_counters;
+  size_t seq_len, cum_thin, thin_tile_base, error, v_thin_base, score_counters, decode_counters;
   size_t score_partials, decode_records, total;
+  size_t value_counters, value_partials;   // value-channel scoring (only with lambda_v > 0)
   size_t header_bytes;     // everything before score_partials (initialised by thinK_create)
 };
 
 struct Geometry {
   int B, L, N_q, N_kv, D, G, T, Tp, S_obs, S_max, R, max_new, cap, tail_tiles_cap, E, dtype, criterion;
   int NC, CB, ncolblk, RPmax;
+  // value-channel pruning (App. D)
+  bool vt;
+  int Tv, Tvp;                 // kept value channels, padded to a multiple of 16
+  int M, MB, nrb;              // query rows per unit of the value score, rows per row block, row blocks
+  int value_slots;             // partial records the workspace holds
+  int S_pmax;
+  std::vector<int64_t> v_thin_base;   // element offsets per batch entry (+ total)
   int64_t total_thin_tiles;    // over all (b, l, h)
   int max_thin_tiles;          // per (l, h) over b
   std::vector<int32_t> seq_len, cum_thin;
@@ -64,6 +72,29 @@ thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geome
     if (nt > g->max_thin_tiles) g->max_thin_tiles = nt;
   }
   g->total_thin_tiles = g->thin_tile_base[c->B];
+  // value channels
+  if (!(c->lambda_v >= 0.0 && c->lambda_v < 1.0)) return THINK_ERR_INVALID_ARG;
+  g->vt = c->lambda_v > 0.0;
+  g->Tv = thinK_T(c->lambda_v, c->D);
+  if (g->Tv < 1) return THINK_ERR_INVALID_ARG;
+  g->Tvp = (g->Tv + 15) & ~15;
+  g->M = g->G * c->S_obs;
+  g->MB = g->M < 128 ? (g->M + 15) & ~15 : 128;
+  g->nrb = (g->M + g->MB - 1) / g->MB;
+  g->value_slots = 0;
+  g->S_pmax = 0;
+  g->v_thin_base.assign(c->B + 1, 0);
+  if (g->vt) {
+    if (c->dtype != THINK_BF16) return THINK_ERR_UNSUPPORTED;
+    if (g->M > 2048) return THINK_ERR_UNSUPPORTED;
+    const int per_layer = c->B * c->N_kv * g->nrb;
+    g->value_slots = per_layer > 4 * kSMs ? per_layer : 4 * kSMs;
+    for (int b = 0; b < c->B; ++b) {
+      const int S_p = seq_lens[b] - c->S_recent;
+      if (S_p > g->S_pmax) g->S_pmax = S_p;
+      g->v_thin_base[b + 1] = g->v_thin_base[b] + (int64_t)c->L * c->N_kv * S_p * g->Tvp;
+    }
+  }
   return THINK_OK;
 }
 
@@ -73,8 +104,11 @@ void make_layout(const Geometry& g, Layout* w) {
   w->cum_thin = o;         o = align_up(o + sizeof(int32_t) * (g.B + 1), 256);
   w->thin_tile_base = o;   o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
   w->error = o;            o = align_up(o + 256, 256);
+  w->v_thin_base = o;      o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
   w->score_counters = o;   o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.ncolblk, 256);
   w->decode_counters = o;  o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.N_kv, 256);
+  w->value_counters = o;
+  if (g.vt) o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.N_kv, 256);   // zeroed with the header
   w->header_bytes = o;
   w->score_partials = o;
   // a call splits tokens so that items * nsplit <= target + items
@@ -82,6 +116,8 @@ void make_layout(const Geometry& g, Layout* w) {
   o = align_up(o + slots * 2 * (size_t)g.CB * (16 / g.E) * sizeof(double), 256);
   w->decode_records = o;
   o = align_up(o + (size_t)kMaxDecodeCtas * 2 * decode_record_bytes(g.D, g.G), 256);
+  w->value_partials = o;
+  if (g.vt) o = align_up(o + (size_t)g.value_slots * score_value_record_bytes(g.MB, g.D), 256);
   w->total = o;
 }
 
@@ -104,7 +140,9 @@ struct thinK_cache {
   Layout w;
   unsigned char* ws;
   void *k_thin, *tail_k, *tail_v, *idx, *scores;
+  void *v_thin, *perm_v, *scores_v;         // value-channel pruning (attached separately)
   std::vector<uint8_t> scored, compacted;   // per layer
+  std::vector<uint8_t> scored_v;            // per layer: value channels ranked
   std::vector<int32_t> tail_len;            // per layer, tokens in the tail buffers
   std::vector<int32_t> n_re;                // per layer, 64-token tail blocks already re-pruned
   thinK_tensor5 v;                          // borrowed prompt values (set by thinK_compact)
@@ -155,6 +193,14 @@ thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens,
     think_elems += S_p * g.T + (size_t)(g.R + new_tokens) * g.D + (S + new_tokens) * g.D;
     dense_elems += 2 * (S + new_tokens) * g.D;
   }
+  out->v_thin = out->perm_v = 0;
+  if (g.vt) {
+    out->v_thin = align_up((size_t)g.v_thin_base[g.B] * g.E, 256);
+    if (out->v_thin == 0) out->v_thin = 256;
+    out->perm_v = align_up(units * g.D, 256);
+    // the prefix values shrink to T_v channels as well
+    for (int b = 0; b < g.B; ++b) think_elems -= (size_t)(g.seq_len[b] - g.R) * (g.D - g.Tv);
+  }
   out->model_think_bytes = think_elems * g.L * g.N_kv * g.E;
   out->model_dense_bytes = dense_elems * g.L * g.N_kv * g.E;
   return THINK_OK;
@@ -175,6 +221,8 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
   make_layout(c->g, &c->w);
   c->ws = (unsigned char*)workspace;
   c->k_thin = k_thin; c->tail_k = tail_k; c->tail_v = tail_v; c->idx = idx; c->scores = scores;
+  c->v_thin = c->perm_v = c->scores_v = nullptr;
+  c->scored_v.assign(c->g.L, 0);
   c->scored.assign(c->g.L, 0);
   c->compacted.assign(c->g.L, 0);
   c->tail_len.assign(c->g.L, 0);
@@ -188,6 +236,7 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
   }
   c->num_sms = prop.multiProcessorCount;
   if (decode_setup(c->g.dtype, c->g.D, c->g.G) != cudaSuccess) { delete c; return THINK_ERR_CUDA; }
+  if (c->g.vt && score_value_setup(c->g.D) != cudaSuccess) { delete c; return THINK_ERR_CUDA; }
   int occ = decode_ctas_per_sm(c->g.dtype, c->g.D, c->g.G);
   if (occ < 1) { delete c; return THINK_ERR_CUDA; }
   c->decode_grid_max = c->num_sms * occ;
@@ -201,6 +250,7 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
   ok = ok && cudaMemcpy(c->ws + c->w.seq_len, g.seq_len.data(), sizeof(int32_t) * g.B, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->ws + c->w.cum_thin, g.cum_thin.data(), sizeof(int32_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->ws + c->w.thin_tile_base, g.thin_tile_base.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->ws + c->w.v_thin_base, g.v_thin_base.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   if (!ok) { delete c; return THINK_ERR_CUDA; }
   *out = c;
   return THINK_OK;
@@ -275,7 +325,14 @@ thinK_status compact_impl(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, cons
   if (!check_view(k, g.E) || !check_view(v, g.E)) return THINK_ERR_INVALID_ARG;
   for (int l = layer0; l < layer0 + nlayers; ++l)
     if (!c->scored[l]) return THINK_ERR_STATE;
-  if (c->have_v && memcmp(&c->v, &v_prefix, sizeof(v_prefix)) != 0) return THINK_ERR_INVALID_ARG;  // one V for all layers
+  if (g.vt) {
+    if (tok.rows) return THINK_ERR_UNSUPPORTED;
+    if (!c->v_thin) return THINK_ERR_STATE;
+    for (int l = layer0; l < layer0 + nlayers; ++l)
+      if (!c->scored_v[l]) return THINK_ERR_STATE;
+  } else if (c->have_v && memcmp(&c->v, &v_prefix, sizeof(v_prefix)) != 0) {
+    return THINK_ERR_INVALID_ARG;   // one V for all layers
+  }
   CompactParams p;
   memset(&p, 0, sizeof(p));
   p.tok = tok;
@@ -288,6 +345,19 @@ thinK_status compact_impl(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, cons
   p.re_cap = g.tail_tiles_cap;
   p.layer0 = layer0; p.nlayers = nlayers;
   if (launch_compact(p, g.dtype, g.max_thin_tiles, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  if (g.vt) {
+    CompactValueParams cv;
+    memset(&cv, 0, sizeof(cv));
+    cv.v = to_view(v);
+    cv.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
+    cv.v_thin_base = (const int64_t*)(c->ws + c->w.v_thin_base);
+    cv.perm_v = (const uint8_t*)c->perm_v;
+    cv.v_thin = c->v_thin;
+    cv.B = g.B; cv.L = g.L; cv.N_kv = g.N_kv; cv.D = g.D; cv.Tv = g.Tv; cv.Tvp = g.Tvp; cv.R = g.R;
+    cv.S_pmax = g.S_pmax;
+    cv.layer0 = layer0; cv.nlayers = nlayers;
+    if (launch_compact_value(cv, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  }
   return seed_tail(c, k, v, tok, v_prefix, layer0, nlayers, stream);
 }
 
@@ -299,6 +369,7 @@ thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, const T
     TailWriteParams t;
     memset(&t, 0, sizeof(t));
     t.tok = tok;
+    t.perm_v = g.vt ? (const uint8_t*)c->perm_v : nullptr;
     t.k = to_view(k); t.v = to_view(v);
     t.src_layer_base = 0; t.rows_from_seq_len = 1;
     t.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
@@ -326,6 +397,58 @@ thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int
   return compact_impl(c, k, v, kNoTokenMap, v, layer0, nlayers, stream);
 }
 
+thinK_status thinK_attach_value_cache(thinK_cache* c, void* v_thin, void* perm_v, void* scores_v) {
+  if (!c || !v_thin || !perm_v || !aligned16(v_thin) || !aligned16(perm_v) || (scores_v && !aligned16(scores_v)))
+    return THINK_ERR_INVALID_ARG;
+  if (!c->g.vt) return THINK_ERR_STATE;
+  c->v_thin = v_thin;
+  c->perm_v = perm_v;
+  c->scores_v = scores_v;
+  return THINK_OK;
+}
+
+thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v,
+                                   int32_t layer0, int32_t nlayers, void* stream) {
+  if (!c) return THINK_ERR_INVALID_ARG;
+  if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
+  const Geometry& g = c->g;
+  if (!g.vt || !c->v_thin) return THINK_ERR_STATE;
+  if (!check_view(q_obs, g.E) || !check_view(k, g.E) || !check_view(v, g.E)) return THINK_ERR_INVALID_ARG;
+  thinK_status st = score_select_impl(c, q_obs, k, kNoTokenMap, layer0, nlayers, stream);
+  if (st != THINK_OK) return st;
+  ValueScoreParams p;
+  memset(&p, 0, sizeof(p));
+  p.q = to_view(q_obs); p.k = to_view(k); p.v = to_view(v);
+  p.seq_len = (const int32_t*)(c->ws + c->w.seq_len);
+  p.partials = (float*)(c->ws + c->w.value_partials);
+  p.counters = (uint32_t*)(c->ws + c->w.value_counters);
+  p.perm_v = (uint8_t*)c->perm_v;
+  p.scores_v = (double*)c->scores_v;
+  p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.G = g.G; p.D = g.D; p.Tv = g.Tv; p.S_obs = g.S_obs;
+  p.M = g.M; p.MB = g.MB; p.nrb = g.nrb;
+  // token splits: at least four 64-token tiles each, the finaliser's weights fit its shared memory,
+  // and one launch fills the partial-record slots
+  int min_len = g.seq_len[0];
+  for (int b = 1; b < g.B; ++b) min_len = g.seq_len[b] < min_len ? g.seq_len[b] : min_len;
+  const int per_layer = g.B * g.N_kv * g.nrb;
+  int nsplit = g.value_slots / per_layer;
+  const int by_len = (min_len + kTileTokens - 1) / kTileTokens / 4;
+  if (nsplit > by_len) nsplit = by_len;
+  if (nsplit > 4096 / g.M) nsplit = 4096 / g.M;
+  if (nsplit > 8) nsplit = 8;
+  if (nsplit < 1) nsplit = 1;
+  p.nsplit = nsplit;
+  int per_launch = g.value_slots / (per_layer * nsplit);
+  if (per_launch < 1) per_launch = 1;
+  for (int l0 = layer0; l0 < layer0 + nlayers; l0 += per_launch) {
+    p.layer0 = l0;
+    p.nlayers = l0 + per_launch <= layer0 + nlayers ? per_launch : layer0 + nlayers - l0;
+    if (launch_score_value(p, 32 * (g.MB / 16), (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+  }
+  for (int l = layer0; l < layer0 + nlayers; ++l) c->scored_v[l] = 1;
+  return THINK_OK;
+}
+
 size_t thinK_v_kept_bytes(const thinK_cache* c) {
   if (!c) return 0;
   const Geometry& g = c->g;
@@ -338,6 +461,7 @@ thinK_status thinK_prefill_evicted(thinK_cache* c, thinK_tensor5 q_obs, thinK_te
   if (!c || !v_kept || !aligned16(v_kept)) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   const Geometry& g = c->g;
+  if (g.vt) return THINK_ERR_UNSUPPORTED;
   if (!check_view(v, g.E)) return THINK_ERR_INVALID_ARG;
   TokenMap m;
   thinK_status st = make_token_map(c, tok, tok_stride, src_tokens, &m);
@@ -362,7 +486,9 @@ thinK_status thinK_prefill_evicted(thinK_cache* c, thinK_tensor5 q_obs, thinK_te
 
 thinK_status thinK_prefill(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0,
                            int32_t nlayers, void* stream) {
-  thinK_status st = thinK_score_select(c, q_obs, k, layer0, nlayers, stream);
+  if (!c) return THINK_ERR_INVALID_ARG;
+  thinK_status st = c->g.vt ? thinK_score_select_kv(c, q_obs, k, v, layer0, nlayers, stream)
+                            : thinK_score_select(c, q_obs, k, layer0, nlayers, stream);
   if (st != THINK_OK) return st;
   return thinK_compact(c, k, v, layer0, nlayers, stream);
 }
@@ -382,6 +508,7 @@ thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, 
   TailWriteParams t;
   memset(&t, 0, sizeof(t));
   const int64_t sn = g.D, sl = (int64_t)g.N_kv * g.D, sb = (int64_t)nlayers * sl;
+  t.perm_v = g.vt ? (const uint8_t*)c->perm_v : nullptr;
   t.k = View5{k_new, sb, 0, sl, sn};
   t.v = View5{v_new, sb, 0, sl, sn};
   t.src_layer_base = layer0; t.rows_from_seq_len = 0;
@@ -422,6 +549,12 @@ thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t
   p.n_re = n_re;
   p.n_tail = n_tail;
   p.n_tail_tiles = (n_tail + kTileTokens - 1) / kTileTokens;
+  if (g.vt) {
+    p.v_thin = c->v_thin;
+    p.v_thin_base = (const int64_t*)(c->ws + c->w.v_thin_base);
+    p.perm_v = (const uint8_t*)c->perm_v;
+    p.Tvp = g.Tvp;
+  }
   p.layer0 = layer0; p.nlayers = nlayers;
   p.Ntot = (long long)nlayers * g.N_kv * ((long long)g.cum_thin[g.B] + (long long)g.B * p.n_tail_tiles);
   for (int b = 0; b < g.B; ++b)
@@ -435,7 +568,7 @@ thinK_status thinK_reprune_tail(thinK_cache* c, int32_t keep_recent, int32_t lay
   if (!c || keep_recent < 0) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   const Geometry& g = c->g;
-  if (g.dtype != THINK_BF16) return THINK_ERR_UNSUPPORTED;
+  if (g.dtype != THINK_BF16 || g.vt) return THINK_ERR_UNSUPPORTED;
   const int n_tail = c->tail_len[layer0], n_re = c->n_re[layer0];
   for (int l = layer0; l < layer0 + nlayers; ++l) {
     if (!c->compacted[l]) return THINK_ERR_STATE;

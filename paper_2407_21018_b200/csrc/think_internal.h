@@ -79,8 +79,34 @@ struct GatherRowsParams {    // values of the kept tokens -> dense [B, L, N_kv, 
   int layer0, nlayers;
 };
 
+struct ValueScoreParams {    // App. D: Score_v = column norms of the window's attention output
+  View5 q, k, v;
+  const int32_t* seq_len;
+  float* partials;          // per (unit, row block, split): float m[MB] | float l[MB] | float O[MB][D]
+  uint32_t* counters;       // per unit of the launch
+  uint8_t* perm_v;          // [B, L, N_kv, D]: kept value channels ascending, then the pruned ones ascending
+  double* scores_v;         // [B, L, N_kv, D] or null
+  int B, L, N_kv, G, D, Tv, S_obs;
+  int layer0, nlayers;
+  int M;                    // G * S_obs query rows per unit
+  int MB;                   // rows per row block (multiple of 16, <= 128)
+  int nrb, nsplit;
+};
+
+struct CompactValueParams {  // V_T[t][c] = V[t][perm_v[c]], t < S_p; rows of Tvp elements (zero padded)
+  View5 v;
+  const int32_t* seq_len;
+  const int64_t* v_thin_base;   // element offset of entry b's block in v_thin
+  const uint8_t* perm_v;
+  void* v_thin;
+  int B, L, N_kv, D, Tv, Tvp, R;
+  int S_pmax;                   // longest pruned prefix over the batch
+  int layer0, nlayers;
+};
+
 struct TailWriteParams {
   TokenMap tok;             // applies when rows_from_seq_len is set
+  const uint8_t* perm_v;    // value-channel pruning: tail values are stored in the order perm_v[unit][0..D) (null: as is)
   View5 k, v;               // sources
   int src_layer_base;       // layer index subtracted before applying sl
   int rows_from_seq_len;    // 1: source row = seq_len[b] - R + r ; 0: source row = r
@@ -110,6 +136,12 @@ struct DecodeParams {
   int n_re;                 // of which hold re-pruned tail blocks (64 tokens each, values stay in tail_v)
   int n_tail;               // tokens in the tail buffers (re-pruned blocks included)
   int n_tail_tiles;
+  // value-channel pruning (App. D): prefix values hold Tvp kept channels per row; tail values and the
+  // accumulators use the channel order perm_v[unit][0..D) (kept ascending, then pruned ascending)
+  const void* v_thin;
+  const int64_t* v_thin_base;
+  const uint8_t* perm_v;
+  int Tvp;
   int layer0, nlayers;
   long long Ntot;           // tiles over all units of this call
   int grid;
@@ -121,6 +153,10 @@ int score_ctas_per_sm(int dtype, int criterion);
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s);
 cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_reprune(const RepruneParams& p, cudaStream_t s);
+cudaError_t launch_score_value(const ValueScoreParams& p, int threads, cudaStream_t s);
+cudaError_t score_value_setup(int D);
+size_t score_value_record_bytes(int MB, int D);
+cudaError_t launch_compact_value(const CompactValueParams& p, cudaStream_t s);
 cudaError_t launch_gather_rows(const GatherRowsParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_decode(const DecodeParams& p, int dtype, int D, int G, cudaStream_t s);
 cudaError_t decode_setup(int dtype, int D, int G);   // one-time per-process kernel attributes
@@ -167,6 +203,36 @@ __device__ __forceinline__ int64_t token_row(const TokenMap& m, int64_t unit, in
     return 0;
   }
   return r;
+}
+
+// Rank-count selection of one head by one warp: channel j is kept when fewer than T channels
+// beat it, where k beats j if s[k] > s[j] or (s[k] == s[j] and k < j).  out[0..T) = kept channels
+// ascending; with `rest`, out[T..D) = the other channels ascending (out is then a permutation).
+__device__ __forceinline__ void select_head(const double* s, int D, int T, uint8_t* out, int lane, bool rest) {
+  int base = 0, base_rest = T;
+  for (int j0 = 0; j0 < D; j0 += 32) {
+    int j = j0 + lane;
+    bool keep = false;
+    if (j < D) {
+      double sj = s[j];
+      int rank = 0;
+      for (int k = 0; k < D; ++k) {
+        double sk = s[k];
+        rank += (sk > sj) || (sk == sj && k < j);
+      }
+      keep = rank < T;
+    }
+    const unsigned m = __ballot_sync(0xffffffffu, keep);
+    const unsigned below = (1u << lane) - 1u;
+    if (keep) out[base + __popc(m & below)] = (uint8_t)j;
+    base += __popc(m);
+    if (rest) {
+      const unsigned valid = __ballot_sync(0xffffffffu, j < D);
+      const unsigned o = valid & ~m;
+      if (j < D && !keep) out[base_rest + __popc(o & below)] = (uint8_t)j;
+      base_rest += __popc(o);
+    }
+  }
 }
 
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }

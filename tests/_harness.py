@@ -17,18 +17,22 @@ def to64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to("cpu", torch.float64).numpy()
 
 
-def make_cache(w: wl.Workload, steps=None, criterion=0, keep_scores=True):
+SCORE_V_RTOL = 1e-4                    # value scores: bf16 tensor-core products, softmax weights as hi + lo pairs
+NEAR_TIE_V_REL = 1e-4
+
+
+def make_cache(w: wl.Workload, steps=None, criterion=0, keep_scores=True, lam_v=0.0):
     from paper_2407_21018_b200 import binding as tk
     steps = w.steps if steps is None else steps
     cfg = tk.make_config(w.B, w.L, w.N_q, w.N_kv, w.D, w.S_max, w.S_obs, w.recent, steps, w.lam,
-                         w.torch_dtype, criterion)
+                         w.torch_dtype, criterion, lam_v)
     cache = tk.ThinKCache(cfg, w.seq_lens, device="cuda", keep_scores=keep_scores)
     cache.k_thin.zero_()     # the tiles reserved for re-pruned tail blocks stay unwritten: make buffers comparable
     return cache
 
 
-def make_oracle(w: wl.Workload) -> orc.ThinKOracle:
-    return orc.ThinKOracle(w.B, w.L, w.N_q, w.N_kv, w.D, w.seq_lens, w.S_obs, w.recent, w.lam)
+def make_oracle(w: wl.Workload, lam_v=0.0) -> orc.ThinKOracle:
+    return orc.ThinKOracle(w.B, w.L, w.N_q, w.N_kv, w.D, w.seq_lens, w.S_obs, w.recent, w.lam, lam_v)
 
 
 def bf16_ulp(x: np.ndarray) -> np.ndarray:
@@ -52,30 +56,33 @@ def assert_attn_close(gpu: np.ndarray, want: np.ndarray, dtype: str, where=""):
     return float(err.max())
 
 
-def compare_selection(idx_gpu: np.ndarray, score_gpu, o: orc.ThinKOracle, where=""):
+def compare_selection(idx_gpu: np.ndarray, score_gpu, o: orc.ThinKOracle, where="", values=False):
     """idx bit-exact against the oracle; a head may differ only when the oracle's own scores at
     the cut are a near-tie (relative gap < 1e-6) and the disagreement is confined to channels whose
     scores lie inside that band.  Such heads are counted, and the oracle continues with the GPU's
     choice so that the later comparisons stay element-exact.  Returns the near-tie count."""
     near = 0
     B, L, N = idx_gpu.shape[:3]
+    # values=True: the same comparison for the value channels (App. D), with the tolerance of that kernel
+    o_idx, o_score, T = (o.idx_v, o.score_v, o.T_v) if values else (o.idx, o.score, o.T)
+    s_rtol, band = (SCORE_V_RTOL, NEAR_TIE_V_REL) if values else (SCORE_RTOL, NEAR_TIE_REL)
     for b in range(B):
         for l in range(L):
             for h in range(N):
-                got, want = idx_gpu[b, l, h].astype(np.int64), o.idx[b, l, h]
+                got, want = idx_gpu[b, l, h].astype(np.int64), o_idx[b, l, h]
                 assert (np.diff(got) > 0).all(), f"{where} idx not ascending at {(b, l, h)}"
                 if score_gpu is not None:
-                    np.testing.assert_allclose(score_gpu[b, l, h], o.score[b, l, h], rtol=SCORE_RTOL,
+                    np.testing.assert_allclose(score_gpu[b, l, h], o_score[b, l, h], rtol=s_rtol,
                                                err_msg=f"{where} scores at {(b, l, h)}")
                 if (got == want).all():
                     continue
-                s = o.score[b, l, h]
-                assert orc.near_tie(s, o.T, NEAR_TIE_REL), f"{where} idx mismatch at {(b, l, h)} without a near-tie"
-                cut = np.sort(s)[::-1][o.T - 1]
+                s = o_score[b, l, h]
+                assert orc.near_tie(s, T, band), f"{where} idx mismatch at {(b, l, h)} without a near-tie"
+                cut = np.sort(s)[::-1][T - 1]
                 diff = set(got.tolist()) ^ set(want.tolist())
-                assert all(abs(s[j] - cut) <= 2 * NEAR_TIE_REL * cut for j in diff), \
+                assert all(abs(s[j] - cut) <= 2 * band * cut for j in diff), \
                     f"{where} idx mismatch outside the near-tie band at {(b, l, h)}"
-                o.idx[b, l, h] = got
+                o_idx[b, l, h] = got
                 near += 1
     return near
 
@@ -95,7 +102,13 @@ def compare_cache(cache, o: orc.ThinKOracle, units=None, where=""):
         assert kf.shape[0] == n
         assert (to64(kf) == o.K_full[b][l][h]).all(), f"{where} tail keys differ at {(b, l, h)}"
         S_p = o.K_T[b][l][h].shape[0]
-        assert (to64(vf) == o.V_all[b][l][h][S_p:]).all(), f"{where} tail values differ at {(b, l, h)}"
+        if o.idx_v is None:
+            assert (to64(vf) == o.V_all[b][l][h][S_p:]).all(), f"{where} tail values differ at {(b, l, h)}"
+        else:                      # value channels pruned: V_all holds the unpruned rows only, the prefix is V_T
+            assert (to64(vf) == o.V_all[b][l][h]).all(), f"{where} tail values differ at {(b, l, h)}"
+            vt = to64(tk.v_thin_logical(cache, b, l, h))
+            assert vt.shape == o.V_T[b][l][h].shape and (vt == o.V_T[b][l][h]).all(), \
+                f"{where} V_T differs at {(b, l, h)}"
 
 
 def run_case(w: wl.Workload, steps=None, criterion=0, check_cache=True, fused=False):

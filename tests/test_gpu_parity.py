@@ -189,6 +189,68 @@ def test_eviction_rejects_bad_arguments():
     assert e.value.status == tk.ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("name,S,L,B,lam_v,R", [
+    ("c2", 1100, 2, 1, 0.3, 32),          # GQA 4:1 -> 128 window rows per key head, T_v = 89 (rows padded to 96)
+    ("c4", 600, 1, 3, 0.5, 32),           # MHA -> 32 rows, ragged batch, T_v = 64
+    ("c5", 2100, 1, 1, 0.25, 0),          # S_obs = 64 -> 256 rows = two row blocks; no recent window
+    ("c2", 700, 1, 2, 0.9, 32),           # T_v = 12: one 16-channel group of values
+])
+def test_value_channel_pruning(name, S, L, B, lam_v, R):
+    """App. D through the whole path: value scores and their ranking, thinned prefix values,
+    tail values in the permuted order, decode over thinned keys AND values."""
+    w = dataclasses.replace(wl.shrink(wl.get_config(name), S=S, L=L, B=B, steps=5), S_recent=R)
+    data = wl.make_prefill(w, device="cpu")
+    K, V, Q = data["K"].cuda(), data["V"].cuda(), data["Q_obs"].cuda()
+    cache = make_cache(w, w.steps, lam_v=lam_v)
+    cache.prefill(Q, K, V)
+    torch.cuda.synchronize()
+    o = make_oracle(w, lam_v)
+    K64, V64, Q64 = to64(data["K"]), to64(data["V"]), to64(data["Q_obs"])
+    o.score_select(Q64, K64)
+    o.score_select_v(Q64, K64, V64)
+    compare_selection(cache.idx_tensor().cpu().numpy(), cache.scores_tensor().cpu().numpy(), o, w.name)
+    perm = cache.perm_v_tensor().cpu().numpy()
+    assert (np.sort(perm, axis=-1) == np.arange(w.D)).all(), "perm_v must be a permutation"
+    assert (np.diff(perm[..., o.T_v:].astype(np.int64), axis=-1) > 0).all()
+    near = compare_selection(perm[..., : o.T_v], cache.scores_v_tensor().cpu().numpy(), o, w.name + " values",
+                             values=True)
+    assert near <= max(1, (w.B * w.L * w.N_kv) // 4), f"{near} near-tie heads"
+    o.compact(K64, V64)
+    compare_cache(cache, o, where=w.name)
+    for t in range(w.steps):
+        st = wl.make_step(w, t, device="cpu")
+        cache.append(st["k_new"].cuda(), st["v_new"].cuda())
+        out = cache.decode_attn(st["q"].cuda())
+        torch.cuda.synchronize()
+        o.append(to64(st["k_new"]), to64(st["v_new"]))
+        assert_attn_close(to64(out), o.decode_attn(to64(st["q"])), w.dtype, f"{w.name} step {t}")
+    compare_cache(cache, o, where=w.name + " after decode")
+    assert cache.device_error() == 0
+
+
+def test_value_channel_pruning_state_and_support():
+    from paper_2407_21018_b200 import binding as tk
+    w = wl.shrink(wl.get_config("c2"), S=300, L=1, steps=2)
+    data = wl.make_prefill(w, device="cuda")
+    plain = make_cache(w, 2)
+    with pytest.raises(tk.ThinKError) as e:              # no value pruning configured
+        plain.score_select_kv(data["Q_obs"], data["K"], data["V"])
+    assert e.value.status == tk.ERR_STATE
+    kv = make_cache(w, 2, lam_v=0.5)
+    kv.score_select(data["Q_obs"], data["K"])
+    with pytest.raises(tk.ThinKError) as e:              # value channels not ranked yet
+        kv.compact(data["K"], data["V"])
+    assert e.value.status == tk.ERR_STATE
+    kv.prefill(data["Q_obs"], data["K"], data["V"])
+    with pytest.raises(tk.ThinKError) as e:
+        kv.reprune_tail(0)
+    assert e.value.status == tk.ERR_UNSUPPORTED
+    w32 = wl.shrink(wl.get_config("c1"), S=100, steps=1)
+    with pytest.raises(tk.ThinKError) as e:              # fp32 caches have no value-pruning kernels
+        make_cache(w32, 1, lam_v=0.5)
+    assert e.value.status == tk.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("lam", [0.0, 0.25, 0.75])
 def test_lambda_sweep(lam):
     w = wl.shrink(wl.get_config("c5"), S=1000, L=1, steps=3, lam=lam)
