@@ -38,14 +38,17 @@ FALLBACK_HBM_GBS = 6650.0
 
 
 # --------------------------------------------------------------------------- byte accounting
-def prefill_bytes(w: wl.Workload, T: int) -> int:
+def prefill_bytes(w: wl.Workload, T: int, Tv: int = 0) -> int:
     """Algorithmic bytes of score + select + compact: read K once, read the window queries, write
-    the thinned prefix, the unpruned recent rows (keys and values) and the index list."""
+    the thinned prefix, the unpruned recent rows (keys and values) and the index list.  With value
+    pruning (Tv > 0): V is read once as well and its thinned prefix and channel order are written."""
     e, G, R = w.elem_bytes, w.N_q // w.N_kv, w.recent
     tot = 0
     for S in w.seq_lens:
         S_p = S - R
         per_head = S * w.D * e + w.S_obs * G * w.D * e + S_p * T * e + 2 * R * w.D * e + R * w.D * e + T
+        if Tv:
+            per_head += S_p * w.D * e + S_p * Tv * e + w.D
         tot += per_head * w.L * w.N_kv
     return tot
 
@@ -57,14 +60,16 @@ def prefill_bytes_evicted(w: wl.Workload, T: int) -> int:
     return prefill_bytes(w, T) + sum(S * 4 + 2 * (S - w.recent) * w.D * e for S in w.seq_lens) * w.L * w.N_kv
 
 
-def decode_bytes(w: wl.Workload, T: int, t: int) -> int:
+def decode_bytes(w: wl.Workload, T: int, t: int, Tv: int = 0) -> int:
     """Algorithmic bytes of decode step t (t tokens already appended before it): thinned prefix
-    keys, unpruned tail keys, all values, index list, q in and out."""
+    keys, unpruned tail keys, all values (prefix rows at Tv channels when values are pruned), index
+    list, q in and out."""
     e, R = w.elem_bytes, w.recent
     tot = 0
     for S in w.seq_lens:
         S_p = S - R
-        per_head = S_p * T * e + (R + t + 1) * w.D * e + (S + t + 1) * w.D * e + T
+        values = (S_p * Tv + (R + t + 1) * w.D) * e + w.D if Tv else (S + t + 1) * w.D * e
+        per_head = S_p * T * e + (R + t + 1) * w.D * e + values + T
         tot += per_head * w.L * w.N_kv + 2 * w.L * w.N_q * w.D * e
     return tot
 
@@ -132,8 +137,8 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     w = wl.get_config(args.config)
+    import dataclasses
     if args.lam is not None:
-        import dataclasses
         w = dataclasses.replace(w, lam=args.lam, name=f"{w.name}-lam{args.lam}")
     nsteps = args.decode_steps if args.decode_steps is not None else w.steps
     tok = None
@@ -145,9 +150,13 @@ def run_ours(args):
         data = wl.make_prefill(src, device=dev, pad_nan=False)
     else:
         data = wl.make_prefill(w, device=dev, pad_nan=False)
-    cfg = tk.make_config(w.B, w.L, w.N_q, w.N_kv, w.D, w.S_max, w.S_obs, w.recent, nsteps, w.lam, w.torch_dtype)
+    cfg = tk.make_config(w.B, w.L, w.N_q, w.N_kv, w.D, w.S_max, w.S_obs, w.recent, nsteps, w.lam, w.torch_dtype,
+                         lam_v=args.lam_v)
     cache = tk.ThinKCache(cfg, w.seq_lens, device=dev, keep_scores=True)
     T = cache.T
+    Tv = cache.T_v if args.lam_v > 0 else 0
+    if Tv:
+        w = dataclasses.replace(w, name=f"{w.name}-lamv{args.lam_v}")
 
     K, V, Q = data["K"], data["V"], data["Q_obs"]
     nvar = min(4, max(1, nsteps))
@@ -160,6 +169,9 @@ def run_ours(args):
             ev["p0"].record(stream)
         if tok is not None:
             cache.prefill_evicted(Q, K, V, tok)
+        elif Tv:
+            cache.score_select_kv(Q, K, V)
+            cache.compact(K, V)
         else:
             cache.score_select(Q, K)
             cache.compact(K, V)
@@ -210,9 +222,9 @@ def run_ours(args):
     prefill_ms = [e["p0"].elapsed_time(e["p1"]) for e in evs]
     dec_ms = [[e["d0"][t].elapsed_time(e["d1"][t]) for t in range(nsteps)] for e in evs]
     dec_mean_us = 1e3 * sum(sum(r) for r in dec_ms) / max(1, args.steps * nsteps)
-    dec_bytes = [decode_bytes(w, T, t) for t in range(nsteps)]
+    dec_bytes = [decode_bytes(w, T, t, Tv) for t in range(nsteps)]
     dec_bytes_mean = sum(dec_bytes) / max(1, nsteps)
-    pre_b = prefill_bytes_evicted(w, T) if tok is not None else prefill_bytes(w, T)
+    pre_b = prefill_bytes_evicted(w, T) if tok is not None else prefill_bytes(w, T, Tv)
     pre_us = 1e3 * sum(prefill_ms) / len(prefill_ms)
     pass_bytes = pre_b + sum(dec_bytes) + nsteps * append_bytes(w)
     ms_per_step = total_ms / args.steps
@@ -242,8 +254,7 @@ def run_ours(args):
             if tok is not None:
                 cache.prefill_evicted(Q, K, V, tok)
             else:
-                cache.score_select(Q, K)
-                cache.compact(K, V)
+                cache.prefill(Q, K, V)
             for t in range(nsteps):
                 s = hs[t % nvar]
                 dq.copy_(s["q"], non_blocking=True)
@@ -281,7 +292,8 @@ def run_ours(args):
             "dtype": w.dtype, "data": "synthetic",
             "config": {"workload": f"{w.name}: B={w.B} S={list(w.seq_lens) if len(set(w.seq_lens)) > 1 else w.seq_lens[0]} "
                                    f"L={w.L} heads={w.N_q}q/{w.N_kv}kv D={w.D} S_obs={w.S_obs} S_recent={w.recent} "
-                                   f"lambda={w.lam} T={T} decode_steps={nsteps}",
+                                   f"lambda={w.lam} T={T}" + (f" lambda_v={args.lam_v} T_v={Tv}" if Tv else "") +
+                                   f" decode_steps={nsteps}",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "l2": "inputs larger than L2 (K, V and the caches are each several L2 sizes)"},
             "decode": {"us_per_step": dec_mean_us, "GBps": dec_gbs, "frac_of_measured": dec_gbs / peak,
@@ -296,7 +308,7 @@ def run_ours(args):
                          "traffic": NCU_DECODE_TRAFFIC_BYTES.get(w.name), "traffic_unit": "bytes per launch"},
             "clocks": clocks,
             "e2e": e2e,
-            "gpu_launches": args.steps * (2 + (1 if w.recent > 0 else 0) + (1 if tok is not None else 0) + 2 * nsteps
+            "gpu_launches": args.steps * (2 + (1 if w.recent > 0 else 0) + (1 if tok is not None else 0) + (2 if Tv else 0) + 2 * nsteps
                                           + (nsteps // args.reprune_every if args.reprune_every else 0)),
             "cpu_baseline": cpu,
         }
@@ -390,6 +402,8 @@ def main():
     ap.add_argument("--kv-size", type=int, default=0,
                     help="prefill behind a token-eviction method that kept this many tokens per head "
                          "(thinK_prefill_evicted on seeded kept-token lists); 0 = no eviction")
+    ap.add_argument("--lam-v", type=float, default=0.0,
+                    help="also prune the value channels with this ratio (App. D); 0 = values untouched")
     ap.add_argument("--lam", type=float, default=None, help="override the config's pruning ratio (c5 sweep)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
