@@ -58,6 +58,63 @@ __device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& hi, uin
   sum += (__bfloat162float(h0) + __bfloat162float(l0)) + (__bfloat162float(h1) + __bfloat162float(l1));
 }
 
+// Ticket + finaliser shared by both kernels: the CTA that arrives last for the unit merges the splits
+// row by row (in split order), forms the column norms over all M rows in fp64 and ranks the channels.
+// `smem`: scratch of at least nsplit*M*4 + (kRowGroups + 1)*D*8 bytes, free to overwrite.
+template <int D>
+__device__ void finish_unit(const ValueScoreParams& p, unsigned char* smem, int ucall, int b, int l, int h) {
+  __shared__ int s_last;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x;
+  const size_t rec_floats = (size_t)p.MB * (2 + D);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(p.counters + ucall, 1u) == (uint32_t)(p.nrb * p.nsplit - 1);
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+
+  float* w = (float*)smem;                                   // [nsplit][M]: weight of a split's row / its denominator
+  double* en = (double*)(smem + (((size_t)p.nsplit * p.M * 4 + 15) & ~(size_t)15));   // [kRowGroups][D]
+  double* sc = en + kRowGroups * D;                          // [D]
+  const float* ubase = p.partials + (size_t)ucall * p.nrb * p.nsplit * rec_floats;
+  for (int r = tid; r < p.M; r += nthreads) {
+    const float* rrec = ubase + (size_t)(r / p.MB) * p.nsplit * rec_floats;
+    const int rl = r % p.MB;
+    float mx = -INFINITY;
+    for (int sp = 0; sp < p.nsplit; ++sp) mx = fmaxf(mx, __ldcg(rrec + sp * rec_floats + rl));
+    float den = 0.f;
+    for (int sp = 0; sp < p.nsplit; ++sp)
+      den += __ldcg(rrec + sp * rec_floats + p.MB + rl) * exp2f(__ldcg(rrec + sp * rec_floats + rl) - mx);
+    for (int sp = 0; sp < p.nsplit; ++sp) w[sp * p.M + r] = exp2f(__ldcg(rrec + sp * rec_floats + rl) - mx) / den;
+  }
+  __syncthreads();
+  for (int item = tid; item < kRowGroups * D; item += nthreads) {
+    const int rg = item / D, j = item % D;
+    double e = 0.0;
+    for (int r = rg; r < p.M; r += kRowGroups) {
+      const float* rrec = ubase + (size_t)(r / p.MB) * p.nsplit * rec_floats + 2 * p.MB + (size_t)(r % p.MB) * D + j;
+      float x = 0.f;
+      for (int sp = 0; sp < p.nsplit; ++sp) x = fmaf(__ldcg(rrec + sp * rec_floats), w[sp * p.M + r], x);
+      e = fma((double)x, (double)x, e);
+    }
+    en[rg * D + j] = e;
+  }
+  __syncthreads();
+  for (int j = tid; j < D; j += nthreads) {
+    double e = 0.0;
+    for (int rg = 0; rg < kRowGroups; ++rg) e += en[rg * D + j];
+    sc[j] = sqrt(e);
+  }
+  __syncthreads();
+  const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+  if (warp == 0) {
+    select_head(sc, D, p.Tv, p.perm_v + unit * D, lane, true);
+    if (p.scores_v)
+      for (int j = lane; j < D; j += 32) p.scores_v[unit * D + j] = sc[j];
+  }
+  if (tid == 0) p.counters[ucall] = 0u;   // ready for the next launch
+}
+
 template <int D>
 __global__ void __launch_bounds__(256, 1) k_score_value(const ValueScoreParams p) {
   constexpr int KS = D / 16, NT = D / 8;
@@ -65,7 +122,6 @@ __global__ void __launch_bounds__(256, 1) k_score_value(const ValueScoreParams p
   constexpr int ROWB = D * 2;
   constexpr int kTileBytes = kVTile * ROWB;
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ int s_last;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x;
   const int qd = lane & 3, frow = lane >> 2;
   const int split = blockIdx.x, rb = blockIdx.y, ucall = blockIdx.z;
@@ -210,54 +266,279 @@ __global__ void __launch_bounds__(256, 1) k_score_value(const ValueScoreParams p
       *(float2*)(ob + 8 * t) = make_float2(o[t][2], o[t][3]);
     }
   }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = atomicAdd(p.counters + ucall, 1u) == (uint32_t)(p.nrb * p.nsplit - 1);
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
+  finish_unit<D>(p, smem, ucall, b, l, h);
+}
 
-  // ---- finaliser: merge the splits row by row, column norms over all M rows, ranking
-  float* w = (float*)smem;                                   // [nsplit][M]: weight of a split's row / its denominator
-  double* en = (double*)(smem + (((size_t)p.nsplit * p.M * 4 + 15) & ~(size_t)15));   // [kRowGroups][D]
-  double* sc = en + kRowGroups * D;                          // [D]
-  const float* ubase = p.partials + (size_t)ucall * p.nrb * p.nsplit * rec_floats;
-  for (int r = tid; r < p.M; r += nthreads) {
-    const float* rrec = ubase + (size_t)(r / p.MB) * p.nsplit * rec_floats;
-    const int rl = r % p.MB;
-    float mx = -INFINITY;
-    for (int sp = 0; sp < p.nsplit; ++sp) mx = fmaxf(mx, __ldcg(rrec + sp * rec_floats + rl));
-    float den = 0.f;
-    for (int sp = 0; sp < p.nsplit; ++sp)
-      den += __ldcg(rrec + sp * rec_floats + p.MB + rl) * exp2f(__ldcg(rrec + sp * rec_floats + rl) - mx);
-    for (int sp = 0; sp < p.nsplit; ++sp) w[sp * p.M + r] = exp2f(__ldcg(rrec + sp * rec_floats + rl) - mx) / den;
-  }
-  __syncthreads();
-  for (int item = tid; item < kRowGroups * D; item += nthreads) {
-    const int rg = item / D, j = item % D;
-    double e = 0.0;
-    for (int r = rg; r < p.M; r += kRowGroups) {
-      const float* rrec = ubase + (size_t)(r / p.MB) * p.nsplit * rec_floats + 2 * p.MB + (size_t)(r % p.MB) * D + j;
-      float x = 0.f;
-      for (int sp = 0; sp < p.nsplit; ++sp) x = fmaf(__ldcg(rrec + sp * rec_floats), w[sp * p.M + r], x);
-      e = fma((double)x, (double)x, e);
-    }
-    en[rg * D + j] = e;
-  }
-  __syncthreads();
-  for (int j = tid; j < D; j += nthreads) {
-    double e = 0.0;
-    for (int rg = 0; rg < kRowGroups; ++rg) e += en[rg * D + j];
-    sc[j] = sqrt(e);
-  }
-  __syncthreads();
-  const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+// ---------------------------------------------------------------------------------------------
+// The same computation on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
+// memory), for D = 128 and blocks of 128 query rows.  A CTA of 128 threads owns (token split, row
+// block, unit); thread t owns query row t = tensor-memory lane t.
+//   per tile of 64 tokens:   S = Q K^T      one thread issues 8 MMAs (M128 N64 K16), S in TMEM columns [0, 64)
+//                            softmax        every thread reads its row of S, writes P = hi + lo as bf16 rows
+//                            O += P V       one thread issues 4 + 4 MMAs (M128 N128 K16), O in columns [64, 192)
+// Operands sit in shared memory in the canonical 128-byte-swizzled layouts (rows of 128 bytes, 16-byte
+// chunk index XOR row%8, 1024-byte groups of 8 rows): Q, K and P K-major, V MN-major -- which is exactly
+// V's natural [token][channel] order, so no transpose is needed.  The running maximum is only raised when it
+// grows by more than 8 (in the exp2 domain): O in tensor memory is then rescaled, otherwise the stale
+// maximum stays and numerator and denominator simply carry the same bounded factor.
+// K(t+1) is fetched while tile t is in its softmax and second product, V(t+1) during the first product and
+// softmax of tile t+1; two CTAs per SM overlap the rest.  Every wait on an mbarrier is bounded: on a
+// time-out the CTA raises the error word, releases its tensor memory and leaves without a ticket.
+// ---------------------------------------------------------------------------------------------
+constexpr int kTcThreads = 128;
+constexpr int kTcQ = 0, kTcK = 32768, kTcV = 49152, kTcPhi = 65536, kTcPlo = 81920, kTcBytes = 98304;
+constexpr int kTcCols = 256;              // allocated tensor-memory columns (power of two): S 64 + O 128
+constexpr uint32_t kTcColO = 64;
+// instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128; N and the majorness of B differ
+constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+// shared-memory matrix descriptor, 128-byte swizzle: address, leading and stride byte offsets in 16-byte units
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((saddr >> 4) & 0x3fffu) | ((uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16) |
+         ((uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32) | (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t"
+      "}\n"
+      :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t"
+      "}\n"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait (about a second): false on time-out
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try(bar, parity))
+    if (clock64() - t0 > 2000000000LL) return false;
+  return true;
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};\n"
+      :: "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+         "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+         "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueScoreParams p) {
+  constexpr int D = 128;
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) uint64_t s_bar[2];
+  __shared__ uint32_t s_tmem;
+  const uint32_t sraw = smem_u32(smem_raw), sb = (sraw + 1023u) & ~1023u;   // swizzle atoms want 1024-byte alignment
+  unsigned char* smem = smem_raw + (sb - sraw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int split = blockIdx.x, rb = blockIdx.y, ucall = blockIdx.z;
+  const int h = ucall % p.N_kv, bl = ucall / p.N_kv;
+  const int ll = bl % p.nlayers, b = bl / p.nlayers, l = p.layer0 + ll;
+  const int S_b = p.seq_len[b];
+  const int ntile_all = (S_b + kVTile - 1) / kVTile;
+  const int per = (ntile_all + p.nsplit - 1) / p.nsplit;
+  const int t0 = min(S_b, split * per * kVTile), t1 = min(S_b, (split + 1) * per * kVTile);
+  const int ntl = (t1 - t0 + kVTile - 1) / kVTile;
+  const uint32_t bar_s = smem_u32(&s_bar[0]), bar_o = smem_u32(&s_bar[1]);
+
   if (warp == 0) {
-    select_head(sc, D, p.Tv, p.perm_v + unit * D, lane, true);
-    if (p.scores_v)
-      for (int j = lane; j < D; j += 32) p.scores_v[unit * D + j] = sc[j];
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(smem_u32(&s_tmem)), "r"(kTcCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (tid == 0) p.counters[ucall] = 0u;   // ready for the next launch
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar_s) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar_o) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+
+  // byte offset of 16-byte chunk ck (0..15) of row r inside an operand made of two 64-element blocks
+  auto swz = [](int r, int ck, int block_bytes) -> uint32_t {
+    return (uint32_t)((ck >> 3) * block_bytes + (r >> 3) * 1024 + (r & 7) * 128 + (((ck & 7) ^ (r & 7)) << 4));
+  };
+  {
+    // query row of this thread: row r of the unit = query head h*G + r / S_obs, window row r % S_obs
+    const int r = rb * p.MB + tid;
+    const bool ok = r < p.M;
+    const __nv_bfloat16* q = (const __nv_bfloat16*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl +
+                             (int64_t)(ok ? r % p.S_obs : 0) * p.q.ss + (int64_t)(h * p.G + (ok ? r / p.S_obs : 0)) * p.q.sn;
+#pragma unroll
+    for (int ck = 0; ck < 16; ++ck) cp_async16_zfill(sb + kTcQ + swz(tid, ck, 16384), q + ck * 8, ok ? 16 : 0);
+    cp_commit();
+  }
+  const __nv_bfloat16* kg = (const __nv_bfloat16*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn;
+  const __nv_bfloat16* vg = (const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;
+  auto load_tile = [&](uint32_t dst, const __nv_bfloat16* g, int64_t stride, int tok0) {
+#pragma unroll
+    for (int i = 0; i < kVTile * 16 / kTcThreads; ++i) {
+      const int idx = tid + i * kTcThreads, r = idx >> 4, ck = idx & 15;
+      const bool ok = tok0 + r < t1;               // rows past the range are zero-filled
+      cp_async16_zfill(dst + swz(r, ck, 8192), g + (int64_t)(ok ? tok0 + r : t0) * stride + ck * 8, ok ? 16 : 0);
+    }
+  };
+  if (ntl > 0) load_tile(sb + kTcK, kg, p.k.ss, t0);
+  cp_commit();
+  if (ntl > 0) load_tile(sb + kTcV, vg, p.v.ss, t0);
+  cp_commit();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  const uint32_t tlane = tmem + ((uint32_t)(warp * 32) << 16);     // this warp's 32 lanes
+
+  const float scale = 1.4426950408889634f / sqrtf((float)D);
+  float m_used = -INFINITY, lsum = 0.f;
+  bool ok_all = true;
+  for (int it = 0; it < ntl; ++it) {
+    cp_wait<1>();                 // K(it) (and Q) have landed; V(it) may still be in flight
+    fence_proxy_async();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        umma_bf16(tmem, umma_desc(sb + kTcQ + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                  umma_desc(sb + kTcK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), kIdescQK, ks > 0);
+      umma_commit(bar_s);
+    }
+    if (!__syncthreads_and(mbar_wait(bar_s, it & 1))) { ok_all = false; break; }
+    tc_fence_after();
+    if (it + 1 < ntl) load_tile(sb + kTcK, kg, p.k.ss, t0 + (it + 1) * kVTile);   // the key buffer is free again
+    cp_commit();
+
+    // ---- this thread's row of S: logits in the exp2 domain, masked past the range
+    uint32_t sr[2][32];
+    tmem_ld32(tlane, sr[0]);
+    tmem_ld32(tlane + 32, sr[1]);
+    tmem_wait_ld();
+    const int nvalid = min(kVTile, t1 - (t0 + it * kVTile));
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 64; ++j) {
+      const float x = j < nvalid ? __uint_as_float(sr[j >> 5][j & 31]) * scale : -INFINITY;
+      sr[j >> 5][j & 31] = __float_as_uint(x);
+      mx = fmaxf(mx, x);
+    }
+    const float m_new = fmaxf(m_used, mx);
+    if (__any_sync(0xffffffffu, m_new > m_used + 8.f)) {
+      // raise the maximum: rescale the denominator and this thread's row of O in tensor memory
+      const float factor = ex2(m_used - m_new);
+      if (it > 0) {
+#pragma unroll 1
+        for (int c0 = 0; c0 < D; c0 += 32) {
+          uint32_t o[32];
+          tmem_ld32(tlane + kTcColO + c0, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
+          tmem_st32(tlane + kTcColO + c0, o);
+        }
+        tmem_wait_st();
+      }
+      lsum *= factor;
+      m_used = m_new;
+    }
+    // ---- P = hi + lo, written as rows of the two A operands
+    const uint32_t prow = (uint32_t)((tid >> 3) * 1024 + (tid & 7) * 128);
+#pragma unroll
+    for (int tc = 0; tc < 8; ++tc) {
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int j = 8 * tc + 2 * e;
+        split_pair(ex2(__uint_as_float(sr[j >> 5][j & 31]) - m_used), ex2(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]) - m_used),
+                   hi[e], lo[e], lsum);
+      }
+      const uint32_t off = prow + ((uint32_t)(tc ^ (tid & 7)) << 4);
+      asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(sb + kTcPhi + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+      asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(sb + kTcPlo + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+    }
+    cp_wait<1>();                 // V(it) has landed; K(it + 1) may still be in flight
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks)
+        umma_bf16(tmem + kTcColO, umma_desc(sb + kTcPhi + ks * 32, 16, 1024), umma_desc(sb + kTcV + ks * 2048, 8192, 1024),
+                  kIdescPV, (it > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks)
+        umma_bf16(tmem + kTcColO, umma_desc(sb + kTcPlo + ks * 32, 16, 1024), umma_desc(sb + kTcV + ks * 2048, 8192, 1024),
+                  kIdescPV, 1u);
+      umma_commit(bar_o);
+    }
+    if (!__syncthreads_and(mbar_wait(bar_o, it & 1))) { ok_all = false; break; }
+    tc_fence_after();
+    if (it + 1 < ntl) load_tile(sb + kTcV, vg, p.v.ss, t0 + (it + 1) * kVTile);   // the value buffer is free again
+    cp_commit();
+  }
+  cp_wait<0>();
+
+  // ---- partial state of this thread's row: (stale maximum, denominator, O row), same record as the other kernel
+  if (ok_all) {
+    const size_t rec_floats = (size_t)p.MB * (2 + D);
+    float* rec = p.partials + ((size_t)(ucall * p.nrb + rb) * p.nsplit + split) * rec_floats;
+    rec[tid] = m_used;
+    rec[p.MB + tid] = lsum;
+    float4* orow = (float4*)(rec + 2 * p.MB + (size_t)tid * D);
+#pragma unroll 1
+    for (int c0 = 0; c0 < D; c0 += 32) {
+      uint32_t o[32];
+      if (ntl > 0) {
+        tmem_ld32(tlane + kTcColO + c0, o);
+        tmem_wait_ld();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) o[j] = 0u;
+      }
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+        orow[c0 / 4 + j] = make_float4(__uint_as_float(o[4 * j]), __uint_as_float(o[4 * j + 1]), __uint_as_float(o[4 * j + 2]),
+                                       __uint_as_float(o[4 * j + 3]));
+    }
+  } else if (tid == 0 && p.error) {
+    atomicOr(p.error, kErrWaitTimeout);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kTcCols) : "memory");
+  if (!ok_all) return;
+  finish_unit<D>(p, smem, ucall, b, l, h);
 }
 
 constexpr int smem_bytes(int D) { return kVStages * 2 * kVTile * D * 2; }
@@ -267,6 +548,10 @@ constexpr int smem_bytes(int D) { return kVStages * 2 * kVTile * D * 2; }
 size_t score_value_record_bytes(int MB, int D) { return (size_t)MB * (2 + D) * sizeof(float); }
 
 cudaError_t score_value_setup(int D) {
+  if (D == 128) {
+    cudaError_t e = cudaFuncSetAttribute(k_score_value_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcBytes + 1024);
+    if (e != cudaSuccess) return e;
+  }
   if (D == 128) return cudaFuncSetAttribute(k_score_value<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128));
   if (D == 64) return cudaFuncSetAttribute(k_score_value<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64));
   return cudaErrorInvalidValue;
@@ -275,6 +560,10 @@ cudaError_t score_value_setup(int D) {
 // threads = 32 * (MB / 16): one warp per 16 query rows of the row block
 cudaError_t launch_score_value(const ValueScoreParams& p, int threads, cudaStream_t s) {
   dim3 grid(p.nsplit, p.nrb, p.B * p.nlayers * p.N_kv);
+  if (p.use_tcgen05 && p.D == 128 && p.MB == 128) {
+    k_score_value_tc<<<grid, kTcThreads, kTcBytes + 1024, s>>>(p);
+    return cudaGetLastError();
+  }
   if (p.D == 128) k_score_value<128><<<grid, threads, smem_bytes(128), s>>>(p);
   else if (p.D == 64) k_score_value<64><<<grid, threads, smem_bytes(64), s>>>(p);
   else return cudaErrorInvalidValue;

@@ -149,6 +149,7 @@ struct thinK_cache {
   bool have_v;
   int num_sms, decode_grid_max;
   int score_capacity;                       // resident CTAs of the score kernel on this device
+  int value_score_tcgen05;                  // 0: keep the mma.sync value-score kernel (THINK_VALUE_SCORE=mma_sync)
 };
 
 extern "C" {
@@ -222,6 +223,10 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
   c->ws = (unsigned char*)workspace;
   c->k_thin = k_thin; c->tail_k = tail_k; c->tail_v = tail_v; c->idx = idx; c->scores = scores;
   c->v_thin = c->perm_v = c->scores_v = nullptr;
+  {
+    const char* e = getenv("THINK_VALUE_SCORE");
+    c->value_score_tcgen05 = !(e && strcmp(e, "mma_sync") == 0);
+  }
   c->scored_v.assign(c->g.L, 0);
   c->scored.assign(c->g.L, 0);
   c->compacted.assign(c->g.L, 0);
@@ -426,6 +431,8 @@ thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_te
   p.scores_v = (double*)c->scores_v;
   p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.G = g.G; p.D = g.D; p.Tv = g.Tv; p.S_obs = g.S_obs;
   p.M = g.M; p.MB = g.MB; p.nrb = g.nrb;
+  p.use_tcgen05 = c->value_score_tcgen05;
+  p.error = (uint32_t*)(c->ws + c->w.error);
   // token splits: at least four 64-token tiles each, the finaliser's weights fit its shared memory,
   // and one launch fills the partial-record slots
   int min_len = g.seq_len[0];

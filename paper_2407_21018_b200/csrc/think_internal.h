@@ -30,6 +30,7 @@ struct TokenMap {
   uint32_t* error;
 };
 constexpr uint32_t kErrTokenRange = 1u;   // device error word: a token index was out of range
+constexpr uint32_t kErrWaitTimeout = 2u;  // device error word: a bounded wait on an mbarrier ran out
 
 struct ScoreParams {
   TokenMap tok;
@@ -91,6 +92,8 @@ struct ValueScoreParams {    // App. D: Score_v = column norms of the window's a
   int M;                    // G * S_obs query rows per unit
   int MB;                   // rows per row block (multiple of 16, <= 128)
   int nrb, nsplit;
+  int use_tcgen05;          // D = 128 and MB = 128: tcgen05.mma kernel instead of the mma.sync one
+  uint32_t* error;          // device error word
 };
 
 struct CompactValueParams {  // V_T[t][c] = V[t][perm_v[c]], t < S_p; rows of Tvp elements (zero padded)
