@@ -218,31 +218,55 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
 }
 
 // Value-channel pruning (paper App. D): V_T[t][c] = V[t][perm_v[c]] for c < T_v, rows of Tvp elements
-// (zero padded), t < S_p.  One thread builds one 16-byte piece of one thinned row.
-__global__ void __launch_bounds__(256) k_compact_value(const CompactValueParams p) {
-  const int cpr = p.Tvp / 8;
-  const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.S_pmax * cpr;
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-    const int ck = i % cpr;
-    int64_t r1 = i / cpr;
-    const int t = r1 % p.S_pmax; r1 /= p.S_pmax;
-    const int h = r1 % p.N_kv; r1 /= p.N_kv;
-    const int l = p.layer0 + (int)(r1 % p.nlayers);
-    const int b = (int)(r1 / p.nlayers);
-    const int S_p = p.seq_len[b] - p.R;
-    if (t >= S_p) continue;
-    const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
-    const uint16_t* src = (const uint16_t*)p.v.ptr + b * p.v.sb + (int64_t)t * p.v.ss + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;
-    const uint8_t* pm = p.perm_v + unit * p.D + ck * 8;
+// (zero padded), t < S_p.  A CTA stages 64 value rows of one head in shared memory (cp.async, padded
+// pitch); a thread then owns one 16-byte piece of the thinned rows -- its eight source channels stay in
+// registers -- and walks down the rows, so consecutive threads write consecutive bytes of v_thin.
+__global__ void __launch_bounds__(128) k_compact_value(const CompactValueParams p) {
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int D = p.D, Tvp = p.Tvp;
+  const int pitch = D * 2 + 16;
+  const int h = blockIdx.y;
+  const int b = blockIdx.z / p.nlayers, l = p.layer0 + blockIdx.z % p.nlayers;
+  const int S_p = p.seq_len[b] - p.R;
+  const int tok0 = blockIdx.x * kTileTokens;
+  if (tok0 >= S_p) return;
+  const int nvalid = min(kTileTokens, S_p - tok0);
+  const int tid = threadIdx.x;
+  const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+  const __nv_bfloat16* src = (const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;
+  const int cpr = D / 8;
+  const uint32_t s_addr = (uint32_t)__cvta_generic_to_shared(smem);
+  for (int i = tid; i < nvalid * cpr; i += 128) {
+    const int r = i / cpr, ck = i % cpr;
+    const void* g = src + (int64_t)(tok0 + r) * p.v.ss + ck * 8;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s_addr + r * pitch + ck * 16), "l"(g) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  // this thread's piece and its source channels (byte offsets inside a staged row; 0xffff = padding)
+  const int cpo = Tvp / 8;                     // pieces per thinned row
+  const int rpp = 128 / cpo;                   // rows per pass
+  const int ck = tid % cpo, r0 = tid / cpo;
+  uint32_t off[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int c = ck * 8 + j;
+    off[j] = c < p.Tv ? 2u * p.perm_v[unit * D + c] : 0xffffu;
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+  if (r0 >= rpp) return;
+  unsigned char* dst = (unsigned char*)p.v_thin +
+                       (p.v_thin_base[b] + ((int64_t)(l * p.N_kv + h) * S_p + tok0) * Tvp) * 2 + ck * 16;
+  for (int r = r0; r < nvalid; r += rpp) {
+    const unsigned char* row = smem + r * pitch;
     uint32_t w[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const int c = ck * 8 + 2 * j;
-      const uint32_t lo = c < p.Tv ? src[pm[2 * j]] : 0u, hi = c + 1 < p.Tv ? src[pm[2 * j + 1]] : 0u;
+      const uint32_t lo = off[2 * j] == 0xffffu ? 0u : *(const uint16_t*)(row + off[2 * j]);
+      const uint32_t hi = off[2 * j + 1] == 0xffffu ? 0u : *(const uint16_t*)(row + off[2 * j + 1]);
       w[j] = lo | (hi << 16);
     }
-    uint16_t* dst = (uint16_t*)p.v_thin + p.v_thin_base[b] + ((int64_t)(l * p.N_kv + h) * S_p + t) * p.Tvp + ck * 8;
-    *(uint4*)dst = make_uint4(w[0], w[1], w[2], w[3]);
+    *(uint4*)(dst + (int64_t)r * Tvp * 2) = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
@@ -270,10 +294,10 @@ __global__ void __launch_bounds__(256) k_gather_rows(const GatherRowsParams p) {
 }  // namespace
 
 cudaError_t launch_compact_value(const CompactValueParams& p, cudaStream_t s) {
-  const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.S_pmax * (p.Tvp / 8);
-  if (total <= 0) return cudaSuccess;
-  const int64_t want = (total + 255) / 256;
-  k_compact_value<<<(int)(want < (int64_t)kSMs * 32 ? want : (int64_t)kSMs * 32), 256, 0, s>>>(p);
+  const int ntiles = (p.S_pmax + kTileTokens - 1) / kTileTokens;
+  if (ntiles <= 0) return cudaSuccess;
+  const size_t smem = (size_t)kTileTokens * (p.D * 2 + 16);
+  k_compact_value<<<dim3(ntiles, p.N_kv, p.B * p.nlayers), 128, smem, s>>>(p);
   return cudaGetLastError();
 }
 

@@ -58,6 +58,14 @@ __device__ __forceinline__ void split_pair(float x0, float x1, uint32_t& hi, uin
   sum += (__bfloat162float(h0) + __bfloat162float(l0)) + (__bfloat162float(h1) + __bfloat162float(l1));
 }
 
+// the same without the running sum: one packed conversion per pair
+__device__ __forceinline__ void split_pair_packed(float x0, float x1, uint32_t& hi, uint32_t& lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  hi = *(const uint32_t*)&h;
+  const __nv_bfloat162 l = __floats2bfloat162_rn(x0 - __uint_as_float(hi << 16), x1 - __uint_as_float(hi & 0xffff0000u));
+  lo = *(const uint32_t*)&l;
+}
+
 // Ticket + finaliser shared by both kernels: the CTA that arrives last for the unit merges the splits
 // row by row (in split order), forms the column norms over all M rows in fp64 and ranks the channels.
 // `smem`: scratch of at least nsplit*M*4 + (kRowGroups + 1)*D*8 bytes, free to overwrite.
@@ -91,11 +99,25 @@ __device__ void finish_unit(const ValueScoreParams& p, unsigned char* smem, int 
   for (int item = tid; item < kRowGroups * D; item += nthreads) {
     const int rg = item / D, j = item % D;
     double e = 0.0;
-    for (int r = rg; r < p.M; r += kRowGroups) {
-      const float* rrec = ubase + (size_t)(r / p.MB) * p.nsplit * rec_floats + 2 * p.MB + (size_t)(r % p.MB) * D + j;
-      float x = 0.f;
-      for (int sp = 0; sp < p.nsplit; ++sp) x = fmaf(__ldcg(rrec + sp * rec_floats), w[sp * p.M + r], x);
-      e = fma((double)x, (double)x, e);
+    // four rows at a time so that their loads are in flight together; sums stay in row order
+    for (int r0 = rg; r0 < p.M; r0 += 4 * kRowGroups) {
+      float x[4] = {0.f, 0.f, 0.f, 0.f};
+      const float* rrec[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int r = min(r0 + u * kRowGroups, p.M - 1);
+        rrec[u] = ubase + (size_t)(r / p.MB) * p.nsplit * rec_floats + 2 * p.MB + (size_t)(r % p.MB) * D + j;
+      }
+      for (int sp = 0; sp < p.nsplit; ++sp) {
+        float v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = __ldcg(rrec[u] + sp * rec_floats);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) x[u] = fmaf(v[u], w[sp * p.M + min(r0 + u * kRowGroups, p.M - 1)], x[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (r0 + u * kRowGroups < p.M) e = fma((double)x[u], (double)x[u], e);
     }
     en[rg * D + j] = e;
   }
@@ -444,14 +466,20 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
     tmem_ld32(tlane + 32, sr[1]);
     tmem_wait_ld();
     const int nvalid = min(kVTile, t1 - (t0 + it * kVTile));
-    float mx = -INFINITY;
+    if (nvalid < kVTile) {        // last tile of the range: tokens past it get weight zero
 #pragma unroll
-    for (int j = 0; j < 64; ++j) {
-      const float x = j < nvalid ? __uint_as_float(sr[j >> 5][j & 31]) * scale : -INFINITY;
-      sr[j >> 5][j & 31] = __float_as_uint(x);
-      mx = fmaxf(mx, x);
+      for (int j = 0; j < 64; ++j)
+        if (j >= nvalid) sr[j >> 5][j & 31] = 0xff800000u;   // -inf
     }
-    const float m_new = fmaxf(m_used, mx);
+    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 64; j += 4) {
+      mx0 = fmaxf(mx0, __uint_as_float(sr[j >> 5][j & 31]));
+      mx1 = fmaxf(mx1, __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]));
+      mx2 = fmaxf(mx2, __uint_as_float(sr[(j + 2) >> 5][(j + 2) & 31]));
+      mx3 = fmaxf(mx3, __uint_as_float(sr[(j + 3) >> 5][(j + 3) & 31]));
+    }
+    const float m_new = fmaxf(m_used, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale);   // scale > 0
     if (__any_sync(0xffffffffu, m_new > m_used + 8.f)) {
       // raise the maximum: rescale the denominator and this thread's row of O in tensor memory
       const float factor = ex2(m_used - m_new);
@@ -472,19 +500,24 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
     }
     // ---- P = hi + lo, written as rows of the two A operands
     const uint32_t prow = (uint32_t)((tid >> 3) * 1024 + (tid & 7) * 128);
+    const float neg_m = -m_used;
+    float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int tc = 0; tc < 8; ++tc) {
       uint32_t hi[4], lo[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int j = 8 * tc + 2 * e;
-        split_pair(ex2(__uint_as_float(sr[j >> 5][j & 31]) - m_used), ex2(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]) - m_used),
-                   hi[e], lo[e], lsum);
+        const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), scale, neg_m));
+        const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), scale, neg_m));
+        ls[e] += p0 + p1;          // the denominator takes the weights before the hi + lo split (2^-17 apart)
+        split_pair_packed(p0, p1, hi[e], lo[e]);
       }
       const uint32_t off = prow + ((uint32_t)(tc ^ (tid & 7)) << 4);
       asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(sb + kTcPhi + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
       asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(sb + kTcPlo + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
     }
+    lsum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
     cp_wait<1>();                 // V(it) has landed; K(it + 1) may still be in flight
     fence_proxy_async();
     tc_fence_before();

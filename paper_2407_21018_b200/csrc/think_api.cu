@@ -87,8 +87,10 @@ thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geome
   if (g->vt) {
     if (c->dtype != THINK_BF16) return THINK_ERR_UNSUPPORTED;
     if (g->M > 2048) return THINK_ERR_UNSUPPORTED;
+    // partial records of the value score: 48 MB worth, at least one layer's
     const int per_layer = c->B * c->N_kv * g->nrb;
-    g->value_slots = per_layer > 4 * kSMs ? per_layer : 4 * kSMs;
+    const size_t by_bytes = ((size_t)48 << 20) / score_value_record_bytes(g->MB, c->D);
+    g->value_slots = (size_t)per_layer > by_bytes ? per_layer : (int)by_bytes;
     for (int b = 0; b < c->B; ++b) {
       const int S_p = seq_lens[b] - c->S_recent;
       if (S_p > g->S_pmax) g->S_pmax = S_p;
@@ -438,15 +440,25 @@ thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_te
   int min_len = g.seq_len[0];
   for (int b = 1; b < g.B; ++b) min_len = g.seq_len[b] < min_len ? g.seq_len[b] : min_len;
   const int per_layer = g.B * g.N_kv * g.nrb;
-  int nsplit = g.value_slots / per_layer;
-  const int by_len = (min_len + kTileTokens - 1) / kTileTokens / 4;
-  if (nsplit > by_len) nsplit = by_len;
-  if (nsplit > 4096 / g.M) nsplit = 4096 / g.M;
-  if (nsplit > 8) nsplit = 8;
-  if (nsplit < 1) nsplit = 1;
-  p.nsplit = nsplit;
-  int per_launch = g.value_slots / (per_layer * nsplit);
+  int per_launch = g.value_slots / per_layer;             // layers per launch
+  if (per_launch > nlayers) per_launch = nlayers;
   if (per_launch < 1) per_launch = 1;
+  int max_split = (min_len + kTileTokens - 1) / kTileTokens / 4;
+  if (max_split > 4096 / g.M) max_split = 4096 / g.M;
+  if (max_split > 8) max_split = 8;
+  if (max_split < 1) max_split = 1;
+  // the split that wastes least of the last wave of CTAs (ties: the smaller split, less to merge)
+  const bool tc = p.use_tcgen05 && g.D == 128 && g.MB == 128;
+  const int resident = c->num_sms * (tc ? 2 : (g.MB >= 128 ? 1 : 2));
+  int nsplit = 1;
+  double best = 0.0;
+  for (int s = 1; s <= max_split; ++s) {
+    const long long ctas = (long long)per_layer * per_launch * s;
+    if (ctas > g.value_slots) break;
+    const double waves = (double)ctas / resident, eff = waves / ceil(waves);
+    if (eff > best + 1e-9) { best = eff; nsplit = s; }
+  }
+  p.nsplit = nsplit;
   for (int l0 = layer0; l0 < layer0 + nlayers; l0 += per_launch) {
     p.layer0 = l0;
     p.nlayers = l0 + per_launch <= layer0 + nlayers ? per_launch : layer0 + nlayers - l0;
