@@ -423,7 +423,7 @@ def test_guard_bytes_untouched():
     assert torch.isfinite(buf[:n].float()).all()
 
 
-def _sampled_full_size(name, units, steps_checked, lam=None):
+def _sampled_full_size(name, units, steps_checked, lam=None, lam_v=0.0):
     """Full-size workload in the launch configuration the benchmark times; the oracle checks
     sampled (b, layer, key head) units: literal + closed-form scores, selection, compacted keys and
     the attention rows of the unit's query heads."""
@@ -432,7 +432,7 @@ def _sampled_full_size(name, units, steps_checked, lam=None):
         w = dataclasses.replace(w, lam=lam)
     data = wl.make_prefill(w, device="cuda")
     K, V, Q = data["K"], data["V"], data["Q_obs"]
-    cache = make_cache(w, max(steps_checked) + 1)
+    cache = make_cache(w, max(steps_checked) + 1, lam_v=lam_v)
     cache.prefill(Q, K, V)           # the launch configuration the benchmark times
     torch.cuda.synchronize()
     assert cache.device_error() == 0
@@ -456,6 +456,18 @@ def _sampled_full_size(name, units, steps_checked, lam=None):
         K_T, K_r = orc.compact_keys(Kh, idx, w.recent)
         assert (to64(tk.k_thin_logical(cache, b, l, h)) == K_T).all()
         heads[(b, l, h)] = dict(idx=idx, K_T=K_T, K_full=K_r, V=Vh)
+        if lam_v > 0:                # value channels (App. D): scores, ranking, thinned prefix rows
+            sv = orc.score_value(Qg, Kh, Vh)
+            np.testing.assert_allclose(cache.scores_v_tensor()[b, l, h].cpu().numpy(), sv, rtol=1e-4)
+            perm = cache.perm_v_tensor()[b, l, h].cpu().numpy().astype(np.int64)
+            assert (np.sort(perm) == np.arange(w.D)).all()
+            idx_v = orc.select_top_T(sv, cache.T_v)
+            if not (idx_v == perm[: cache.T_v]).all():
+                assert orc.near_tie(sv, cache.T_v, 1e-4), f"value idx mismatch at {(b, l, h)}"
+                idx_v = perm[: cache.T_v]
+            S_p = S_b - w.recent
+            assert (to64(tk.v_thin_logical(cache, b, l, h)) == Vh[:S_p][:, idx_v]).all()
+            heads[(b, l, h)].update(idx_v=idx_v, V_T=Vh[:S_p][:, idx_v], V=Vh[S_p:])
     worst = 0.0
     for t in range(max(steps_checked) + 1):
         st = wl.make_step(w, t, device="cuda")
@@ -467,7 +479,11 @@ def _sampled_full_size(name, units, steps_checked, lam=None):
             d["V"] = np.vstack([d["V"], to64(st["v_new"][b, l, h])[None]])
             if t in steps_checked:
                 for g in range(G):
-                    want = orc.decode_attention(to64(st["q"][b, l, h * G + g]), d["K_T"], d["idx"], d["K_full"], d["V"])
+                    qrow = to64(st["q"][b, l, h * G + g])
+                    if lam_v > 0:
+                        want = orc.decode_attention_kv(qrow, d["K_T"], d["idx"], d["K_full"], d["V_T"], d["idx_v"], d["V"])
+                    else:
+                        want = orc.decode_attention(qrow, d["K_T"], d["idx"], d["K_full"], d["V"])
                     worst = max(worst, assert_attn_close(to64(out[b, l, h * G + g]), want, w.dtype, f"{name} {(b, l, h, g)} t={t}"))
         if t in steps_checked:
             assert torch.isfinite(out.float()).all()
@@ -477,6 +493,18 @@ def _sampled_full_size(name, units, steps_checked, lam=None):
 
 def test_c2_full_size_sampled():
     _sampled_full_size("c2", [(0, 0, 0), (0, 13, 5), (0, 31, 7), (0, 7, 2)], {0, 1, 5})
+
+
+def test_c2_full_size_sampled_value_pruning():
+    _sampled_full_size("c2", [(0, 0, 0), (0, 19, 6), (0, 31, 3)], {0, 2}, lam_v=0.3)
+
+
+def test_c4_full_size_sampled_value_pruning():
+    _sampled_full_size("c4", [(0, 0, 0), (15, 31, 31), (9, 20, 4)], {0, 1}, lam_v=0.5)
+
+
+def test_c5_full_size_sampled_value_pruning():
+    _sampled_full_size("c5", [(0, 17, 4)], {0}, lam_v=0.5)
 
 
 def test_c3_full_size_sampled():
