@@ -28,16 +28,6 @@ __device__ __forceinline__ float ex2(float x) { return exp2f(x); }
 template <typename Tin, int N>
 __device__ __forceinline__ void load_row(const Tin* p, float (&v)[N]);
 template <>
-__device__ __forceinline__ void load_row<__nv_bfloat16, 4>(const __nv_bfloat16* p, float (&v)[4]) {
-  uint2 w = __ldg((const uint2*)p);
-  v[0] = bf16lo(w.x); v[1] = bf16hi(w.x); v[2] = bf16lo(w.y); v[3] = bf16hi(w.y);
-}
-template <>
-__device__ __forceinline__ void load_row<__nv_bfloat16, 2>(const __nv_bfloat16* p, float (&v)[2]) {
-  uint32_t w = __ldg((const uint32_t*)p);
-  v[0] = bf16lo(w); v[1] = bf16hi(w);
-}
-template <>
 __device__ __forceinline__ void load_row<float, 4>(const float* p, float (&v)[4]) {
   float4 w = __ldg((const float4*)p);
   v[0] = w.x; v[1] = w.y; v[2] = w.z; v[3] = w.w;
@@ -48,16 +38,11 @@ __device__ __forceinline__ void load_row<float, 2>(const float* p, float (&v)[2]
   v[0] = w.x; v[1] = w.y;
 }
 
-__device__ __forceinline__ void load_pair(const unsigned char* p, float& a, float& b, __nv_bfloat16*) {
-  uint32_t w = __ldg((const uint32_t*)p);
-  a = bf16lo(w); b = bf16hi(w);
-}
 __device__ __forceinline__ void load_pair(const unsigned char* p, float& a, float& b, float*) {
   float2 w = __ldg((const float2*)p);
   a = w.x; b = w.y;
 }
 
-__device__ __forceinline__ void store_out(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 __device__ __forceinline__ void store_out(float* p, float v) { *p = v; }
 
 // CTA that owns flat tile f when N tiles are split over `grid` CTAs as [i*N/grid, (i+1)*N/grid)

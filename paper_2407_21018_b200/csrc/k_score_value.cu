@@ -385,7 +385,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
   __shared__ uint32_t s_tmem;
   const uint32_t sraw = smem_u32(smem_raw), sb = (sraw + 1023u) & ~1023u;   // swizzle atoms want 1024-byte alignment
   unsigned char* smem = smem_raw + (sb - sraw);
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5;
   const int split = blockIdx.x, rb = blockIdx.y, ucall = blockIdx.z;
   const int h = ucall % p.N_kv, bl = ucall / p.N_kv;
   const int ll = bl % p.nlayers, b = bl / p.nlayers, l = p.layer0 + ll;

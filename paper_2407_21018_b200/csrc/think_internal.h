@@ -13,7 +13,6 @@ constexpr int kSMs = 148;             // B200; used only to size the workspace
 constexpr int kScoreThreads = 256;
 constexpr int kScoreTargetCtas = kSMs * 8;
 constexpr int kMaxDecodeCtas = kSMs * 16;
-constexpr int kMaxGroup = 8;
 
 struct View5 {
   const void* ptr;
