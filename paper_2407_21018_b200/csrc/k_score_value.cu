@@ -295,22 +295,23 @@ __global__ void __launch_bounds__(256, 1) k_score_value(const ValueScoreParams p
 // The same computation on the 5th-generation tensor cores (tcgen05.mma, accumulators in tensor
 // memory), for D = 128 and blocks of 128 query rows.  A CTA of 128 threads owns (token split, row
 // block, unit); thread t owns query row t = tensor-memory lane t.
-//   per tile of 64 tokens:   S = Q K^T      one thread issues 8 MMAs (M128 N64 K16), S in TMEM columns [0, 64)
+//   per tile of 64 tokens:   S = Q K^T      one thread issues 8 MMAs (M128 N64 K16), S in TMEM columns [0, 64) or [64, 128)
 //                            softmax        every thread reads its row of S, writes P = hi + lo as bf16 rows
-//                            O += P V       one thread issues 4 + 4 MMAs (M128 N128 K16), O in columns [64, 192)
+//                            O += P V       one thread issues 4 + 4 MMAs (M128 N128 K16), O in columns [128, 256)
 // Operands sit in shared memory in the canonical 128-byte-swizzled layouts (rows of 128 bytes, 16-byte
 // chunk index XOR row%8, 1024-byte groups of 8 rows): Q, K and P K-major, V MN-major -- which is exactly
 // V's natural [token][channel] order, so no transpose is needed.  The running maximum is only raised when it
 // grows by more than 8 (in the exp2 domain): O in tensor memory is then rescaled, otherwise the stale
 // maximum stays and numerator and denominator simply carry the same bounded factor.
-// K(t+1) is fetched while tile t is in its softmax and second product, V(t+1) during the first product and
-// softmax of tile t+1; two CTAs per SM overlap the rest.  Every wait on an mbarrier is bounded: on a
+// K(t+1) is fetched during the softmax of tile t and its first product is issued right behind the second
+// product of tile t (into the other S buffer); V(t+1) is fetched during the softmax of tile t+1; two CTAs
+// per SM overlap the rest.  Every wait on an mbarrier is bounded: on a
 // time-out the CTA raises the error word, releases its tensor memory and leaves without a ticket.
 // ---------------------------------------------------------------------------------------------
 constexpr int kTcThreads = 128;
 constexpr int kTcQ = 0, kTcK = 32768, kTcV = 49152, kTcPhi = 65536, kTcPlo = 81920, kTcBytes = 98304;
-constexpr int kTcCols = 256;              // allocated tensor-memory columns (power of two): S 64 + O 128
-constexpr uint32_t kTcColO = 64;
+constexpr int kTcCols = 256;              // allocated tensor-memory columns (power of two): 2 x S 64 + O 128
+constexpr uint32_t kTcColS1 = 64, kTcColO = 128;   // S buffers at columns 0 and 64, O at 128
 // instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128; N and the majorness of B differ
 constexpr uint32_t kIdescQK = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescPV = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
@@ -443,18 +444,24 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
   const float scale = 1.4426950408889634f / sqrtf((float)D);
   float m_used = -INFINITY, lsum = 0.f;
   bool ok_all = true;
-  for (int it = 0; it < ntl; ++it) {
-    cp_wait<1>();                 // K(it) (and Q) have landed; V(it) may still be in flight
+  // first product of tile `t` into S buffer t & 1 (issued by one thread)
+  auto issue_qk = [&](int t) {
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks)
+      umma_bf16(tmem + (uint32_t)(t & 1) * kTcColS1, umma_desc(sb + kTcQ + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                umma_desc(sb + kTcK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), kIdescQK, ks > 0);
+    umma_commit(bar_s);
+  };
+  if (ntl > 0) {
+    cp_wait<1>();                 // Q and K(0) have landed; V(0) may still be in flight
     fence_proxy_async();
     __syncthreads();
     if (tid == 0) {
       tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
-        umma_bf16(tmem, umma_desc(sb + kTcQ + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                  umma_desc(sb + kTcK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), kIdescQK, ks > 0);
-      umma_commit(bar_s);
+      issue_qk(0);
     }
+  }
+  for (int it = 0; it < ntl; ++it) {
     if (!__syncthreads_and(mbar_wait(bar_s, it & 1))) { ok_all = false; break; }
     tc_fence_after();
     if (it + 1 < ntl) load_tile(sb + kTcK, kg, p.k.ss, t0 + (it + 1) * kVTile);   // the key buffer is free again
@@ -462,8 +469,9 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
 
     // ---- this thread's row of S: logits in the exp2 domain, masked past the range
     uint32_t sr[2][32];
-    tmem_ld32(tlane, sr[0]);
-    tmem_ld32(tlane + 32, sr[1]);
+    const uint32_t tS = tlane + (uint32_t)(it & 1) * kTcColS1;
+    tmem_ld32(tS, sr[0]);
+    tmem_ld32(tS + 32, sr[1]);
     tmem_wait_ld();
     const int nvalid = min(kVTile, t1 - (t0 + it * kVTile));
     if (nvalid < kVTile) {        // last tile of the range: tokens past it get weight zero
@@ -518,7 +526,7 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
       asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(sb + kTcPlo + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
     }
     lsum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-    cp_wait<1>();                 // V(it) has landed; K(it + 1) may still be in flight
+    cp_wait<0>();                 // V(it) and K(it + 1) have landed
     fence_proxy_async();
     tc_fence_before();
     __syncthreads();
@@ -533,6 +541,9 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
         umma_bf16(tmem + kTcColO, umma_desc(sb + kTcPlo + ks * 32, 16, 1024), umma_desc(sb + kTcV + ks * 2048, 8192, 1024),
                   kIdescPV, 1u);
       umma_commit(bar_o);
+      // the next tile's first product goes to the other S buffer right behind it: its round trip hides
+      // behind this tile's second product instead of adding to it
+      if (it + 1 < ntl) issue_qk(it + 1);
     }
     if (!__syncthreads_and(mbar_wait(bar_o, it & 1))) { ok_all = false; break; }
     tc_fence_after();
