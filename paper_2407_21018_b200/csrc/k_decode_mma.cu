@@ -446,18 +446,31 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
         float Lsum = 0.f, acc[EPL];
 #pragma unroll
         for (int k = 0; k < EPL; ++k) acc[k] = 0.f;
-        for (int ci = c_first; ci <= c_last; ++ci) {
-          const uint8_t* r = rec_of(ci);
-          float ov[EPL];
+        // two contributors per trip: both sets of loads are in flight together, sums stay in worker order
+        for (int ci = c_first; ci <= c_last; ci += 2) {
+          const bool two = ci + 1 <= c_last;
+          const uint8_t* r0 = rec_of(ci);
+          const uint8_t* r1 = rec_of(two ? ci + 1 : ci);
+          float ov0[EPL], ov1[EPL];
 #pragma unroll
-          for (int k = 0; k < EPL; ++k) ov[k] = __ldcg((const float*)(r + rec_o_off(G)) + lane + 32 * k);
-          float w = 0.f;
+          for (int k = 0; k < EPL; ++k) ov0[k] = __ldcg((const float*)(r0 + rec_o_off(G)) + lane + 32 * k);
+#pragma unroll
+          for (int k = 0; k < EPL; ++k) ov1[k] = __ldcg((const float*)(r1 + rec_o_off(G)) + lane + 32 * k);
+          float w0 = 0.f, w1 = 0.f;
           if (lane < G) {
-            w = exp2f((float)__ldcg((const double*)r + lane) - M);
-            Lsum += __ldcg((const float*)(r + G * 8) + lane) * w;
+            const float m0 = (float)__ldcg((const double*)r0 + lane), m1 = (float)__ldcg((const double*)r1 + lane);
+            const float l0 = __ldcg((const float*)(r0 + G * 8) + lane), l1 = __ldcg((const float*)(r1 + G * 8) + lane);
+            w0 = exp2f(m0 - M);
+            Lsum += l0 * w0;
+            if (two) {
+              w1 = exp2f(m1 - M);
+              Lsum += l1 * w1;
+            }
           }
 #pragma unroll
-          for (int k = 0; k < EPL; ++k) acc[k] = fmaf(ov[k], __shfl_sync(0xffffffffu, w, (lane + 32 * k) / D), acc[k]);
+          for (int k = 0; k < EPL; ++k) acc[k] = fmaf(ov0[k], __shfl_sync(0xffffffffu, w0, (lane + 32 * k) / D), acc[k]);
+#pragma unroll
+          for (int k = 0; k < EPL; ++k) acc[k] = fmaf(ov1[k], __shfl_sync(0xffffffffu, w1, (lane + 32 * k) / D), acc[k]);
         }
 #pragma unroll
         for (int k = 0; k < EPL; ++k) {
