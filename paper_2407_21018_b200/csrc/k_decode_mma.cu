@@ -103,6 +103,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
   static_assert(D == 64 || D == 128, "head dimension");
   constexpr int NT = D / 8;              // n-tiles of the output
   constexpr int KS = D / 16;             // 16-channel groups of a full key
+  constexpr int kQScratch = G * D * 2 + 128;          // per warp: the group's query rows + the unit's index list
   extern __shared__ __align__(128) unsigned char smem[];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int qd = lane & 3, row = lane >> 2;          // fragment coordinates: row = query head
@@ -286,20 +287,38 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
     }
 
     // ---- query fragments (A operand): qa[s][0] = channels 16s+2qd,+1 ; qa[s][1] = channels 16s+2qd+8,+9
+    // The group's G query rows (contiguous) and the unit's index list go to this warp's scratch in ONE round
+    // trip of independent loads; both the gathered and the full query fragments are then read from there, so a
+    // segment pays one global latency instead of three (index list -> gathered query -> full query).
     const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q + ((int64_t)(b * p.nlayers + ll) * p.N_q + h * G) * D;
     const uint8_t* idx = p.idx + unit_abs * p.T;
+    unsigned char* qs = smem + kSmemBytes + warp * kQScratch;
+    {
+      constexpr int QV = (G * D / 8 + 31) / 32;        // 16-byte pieces of the query rows per lane
+      uint4 qv[QV];
+      uint8_t iv[4];
+#pragma unroll
+      for (int i = 0; i < QV; ++i)
+        if (lane + 32 * i < G * D / 8) qv[i] = __ldg((const uint4*)qg + lane + 32 * i);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) iv[i] = lane + 32 * i < p.T ? idx[lane + 32 * i] : (uint8_t)0;
+      __syncwarp();                                     // the previous segment's readers are done
+#pragma unroll
+      for (int i = 0; i < QV; ++i)
+        if (lane + 32 * i < G * D / 8) ((uint4*)qs)[lane + 32 * i] = qv[i];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) qs[G * D * 2 + lane + 32 * i] = iv[i];
+      __syncwarp();
+    }
     uint32_t qa[KS][2];
     uint32_t qa8 = 0;
     auto q_pair = [&](int c, bool thin) -> uint32_t {   // (q[c], q[c+1]) of this lane's query head
       if (row >= G) return 0u;
-      const uint16_t* qr = (const uint16_t*)(qg + row * D);
-      uint32_t a = 0, bb = 0;
-      if (thin) {
-        if (c < p.T) a = qr[idx[c]];
-        if (c + 1 < p.T) bb = qr[idx[c + 1]];
-      } else {
-        a = qr[c]; bb = qr[c + 1];
-      }
+      const unsigned char* qr = qs + row * (D * 2);
+      if (!thin) return *(const uint32_t*)(qr + 2 * c);
+      const uint8_t* ix = qs + G * D * 2;
+      const uint32_t a = c < p.T ? *(const uint16_t*)(qr + 2 * ix[c]) : 0u;
+      const uint32_t bb = c + 1 < p.T ? *(const uint16_t*)(qr + 2 * ix[c + 1]) : 0u;
       return a | (bb << 16);
     };
     auto load_q = [&](bool thin) {
@@ -489,15 +508,18 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
 
 template <int D, int G>
 cudaError_t launch_mma(const DecodeParams& p, cudaStream_t s) {
-  if (p.v_thin) k_decode_mma<D, G, true><<<p.grid, kWarps * 32, kSmemBytes, s>>>(p);
-  else k_decode_mma<D, G, false><<<p.grid, kWarps * 32, kSmemBytes, s>>>(p);
+  constexpr int smem = kSmemBytes + kWarps * (G * D * 2 + 128);
+  if (p.v_thin) k_decode_mma<D, G, true><<<p.grid, kWarps * 32, smem, s>>>(p);
+  else k_decode_mma<D, G, false><<<p.grid, kWarps * 32, smem, s>>>(p);
   return cudaGetLastError();
 }
 template <int D, int G>
 cudaError_t setup_mma() {
-  cudaError_t e = cudaFuncSetAttribute(k_decode_mma<D, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  constexpr int smem = kSmemBytes + kWarps * (G * D * 2 + 128);
+  static_assert(smem <= 227 * 1024, "ring + query scratch exceed the shared memory of a CTA");
+  cudaError_t e = cudaFuncSetAttribute(k_decode_mma<D, G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_decode_mma<D, G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  return cudaFuncSetAttribute(k_decode_mma<D, G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
 }
 
 #define THINK_MMA_DISPATCH(FN, ...)                                   \
