@@ -31,7 +31,7 @@ from paper_2407_21018_b200 import workloads as wl  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) of ONE launch of the decode kernel from an ncu capture of the current
 # kernel (profiles/k_decode_mma_c2_ncu.md); configs without a capture report null.
-NCU_DECODE_TRAFFIC_BYTES = {"c2": 882.2e6}
+NCU_DECODE_TRAFFIC_BYTES = {"c2": 879.9e6}
 # DRAM bytes of the prefill kernels of one pass (score + compact; profiles/k_*_c2_ncu.md): K crosses HBM twice.
 NCU_PREFILL_TRAFFIC_BYTES = {"c2": 1379.9e6}
 FALLBACK_HBM_GBS = 6650.0
