@@ -222,6 +222,8 @@ def run_ours(args):
     prefill_ms = [e["p0"].elapsed_time(e["p1"]) for e in evs]
     dec_ms = [[e["d0"][t].elapsed_time(e["d1"][t]) for t in range(nsteps)] for e in evs]
     dec_mean_us = 1e3 * sum(sum(r) for r in dec_ms) / max(1, args.steps * nsteps)
+    dec_all = sorted(1e3 * x for r in dec_ms for x in r) or [0.0]
+    pre_all = sorted(1e3 * x for x in prefill_ms)
     dec_bytes = [decode_bytes(w, T, t, Tv) for t in range(nsteps)]
     dec_bytes_mean = sum(dec_bytes) / max(1, nsteps)
     pre_b = prefill_bytes_evicted(w, T) if tok is not None else prefill_bytes(w, T, Tv)
@@ -296,9 +298,10 @@ def run_ours(args):
                                    f" decode_steps={nsteps}",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "l2": "inputs larger than L2 (K, V and the caches are each several L2 sizes)"},
-            "decode": {"us_per_step": dec_mean_us, "GBps": dec_gbs, "frac_of_measured": dec_gbs / peak,
+            "decode": {"us_per_step": dec_mean_us, "us_median": dec_all[len(dec_all) // 2], "us_min": dec_all[0],
+                       "GBps": dec_gbs, "frac_of_measured": dec_gbs / peak,
                        "frac_of_nominal_8TBps": dec_gbs / NOMINAL_HBM_GBS, "bytes_per_step": dec_bytes_mean},
-            "prefill": {"us": pre_us, "GBps": pre_gbs, "frac_of_measured": pre_gbs / peak,
+            "prefill": {"us": pre_us, "us_median": pre_all[len(pre_all) // 2], "us_min": pre_all[0], "GBps": pre_gbs, "frac_of_measured": pre_gbs / peak,
                         "frac_of_nominal_8TBps": pre_gbs / NOMINAL_HBM_GBS, "bytes": pre_b,
                         "dram_bytes_ncu": NCU_PREFILL_TRAFFIC_BYTES.get(w.name),
                         "dram_GBps": (NCU_PREFILL_TRAFFIC_BYTES[w.name] / (pre_us * 1e-6) / 1e9
