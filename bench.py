@@ -179,6 +179,14 @@ def run_ours(args):
             ev["p1"].record(stream)
         for t in range(nsteps):
             s = steps_in[t % nvar]
+            if ev is not None:
+                ev["s0"][t].record(stream)
+            if args.fused_step:
+                cache.append_decode(s["k_new"], s["v_new"], s["q"], out=out)   # one call, overlapped launches
+                if ev is not None:
+                    ev["d0"][t].record(stream)     # (no separate attention time in this mode)
+                    ev["d1"][t].record(stream)
+                continue
             cache.append(s["k_new"], s["v_new"])
             if args.reprune_every and (t + 1) % args.reprune_every == 0:
                 cache.reprune_tail(w.recent)       # App. C.1 control flow: thin the oldest tail blocks
@@ -190,7 +198,8 @@ def run_ours(args):
 
     def mk_events():
         E = lambda: torch.cuda.Event(enable_timing=True)
-        return {"p0": E(), "p1": E(), "d0": [E() for _ in range(nsteps)], "d1": [E() for _ in range(nsteps)]}
+        return {"p0": E(), "p1": E(), "d0": [E() for _ in range(nsteps)], "d1": [E() for _ in range(nsteps)],
+                "s0": [E() for _ in range(nsteps)]}
 
     n_warm = args.warmup if args.profile else max(3, args.warmup)
     for _ in range(n_warm):
@@ -221,6 +230,10 @@ def run_ours(args):
 
     prefill_ms = [e["p0"].elapsed_time(e["p1"]) for e in evs]
     dec_ms = [[e["d0"][t].elapsed_time(e["d1"][t]) for t in range(nsteps)] for e in evs]
+    # whole decode step (append + attention), whichever way it was launched
+    step_us = 1e3 * sum(e["s0"][t].elapsed_time(e["d1"][t]) for e in evs for t in range(nsteps)) / max(1, args.steps * nsteps)
+    if args.fused_step:
+        dec_ms = [[e["s0"][t].elapsed_time(e["d1"][t]) for t in range(nsteps)] for e in evs]
     dec_mean_us = 1e3 * sum(sum(r) for r in dec_ms) / max(1, args.steps * nsteps)
     dec_all = sorted(1e3 * x for r in dec_ms for x in r) or [0.0]
     pre_all = sorted(1e3 * x for x in prefill_ms)
@@ -239,6 +252,25 @@ def run_ours(args):
         peak, peak_src = FALLBACK_HBM_GBS, "fallback"
     dec_gbs = dec_bytes_mean / (dec_mean_us * 1e-6) / 1e9 if nsteps else 0.0
     pre_gbs = pre_b / (pre_us * 1e-6) / 1e9
+
+    # ---- the same pass with thinK_append_decode (one call per decode step, attention overlapped with the append):
+    # reported next to the headline, which keeps the two calls apart so that the attention kernel can be timed alone
+    fused = None
+    if not args.fused_step and nsteps > 0 and not args.reprune_every:
+        saved, args.fused_step = args.fused_step, True
+        one_pass()
+        torch.cuda.synchronize()
+        fa, fb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fev = [mk_events() for _ in range(3)]
+        fa.record(stream)
+        for e in fev:
+            one_pass(e)
+        fb.record(stream)
+        torch.cuda.synchronize()
+        args.fused_step = saved
+        f_ms = fa.elapsed_time(fb) / len(fev)
+        f_step = 1e3 * sum(e["s0"][t].elapsed_time(e["d1"][t]) for e in fev for t in range(nsteps)) / (len(fev) * nsteps)
+        fused = {"ms_per_pass": f_ms, "value_GBps": pass_bytes / (f_ms * 1e-3) / 1e9, "step_us_append_plus_attn": f_step}
 
     # ---- end to end: inputs start in pinned host memory, results are read back every step
     e2e = None
@@ -298,7 +330,8 @@ def run_ours(args):
                                    f" decode_steps={nsteps}",
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "l2": "inputs larger than L2 (K, V and the caches are each several L2 sizes)"},
-            "decode": {"us_per_step": dec_mean_us, "us_median": dec_all[len(dec_all) // 2], "us_min": dec_all[0],
+            "decode": {"step_us_append_plus_attn": step_us, "fused_step": bool(args.fused_step),
+                       "us_per_step": dec_mean_us, "us_median": dec_all[len(dec_all) // 2], "us_min": dec_all[0],
                        "GBps": dec_gbs, "frac_of_measured": dec_gbs / peak,
                        "frac_of_nominal_8TBps": dec_gbs / NOMINAL_HBM_GBS, "bytes_per_step": dec_bytes_mean},
             "prefill": {"us": pre_us, "us_median": pre_all[len(pre_all) // 2], "us_min": pre_all[0], "GBps": pre_gbs, "frac_of_measured": pre_gbs / peak,
@@ -309,6 +342,7 @@ def run_ours(args):
             "roofline": {"kernel": "k_decode_mma" if w.dtype == "bf16" else "k_decode_generic", "bound": "hbm", "achieved": dec_gbs, "peak": peak,
                          "peak_source": f"of {peak_src}", "unit": "GB/s", "frac": dec_gbs / peak,
                          "traffic": NCU_DECODE_TRAFFIC_BYTES.get(w.name), "traffic_unit": "bytes per launch"},
+            "fused_step_variant": fused,
             "clocks": clocks,
             "e2e": e2e,
             "gpu_launches": args.steps * (2 + (1 if w.recent > 0 else 0) + (1 if tok is not None else 0) + (2 if Tv else 0) + 2 * nsteps
@@ -407,6 +441,9 @@ def main():
                          "(thinK_prefill_evicted on seeded kept-token lists); 0 = no eviction")
     ap.add_argument("--lam-v", type=float, default=0.0,
                     help="also prune the value channels with this ratio (App. D); 0 = values untouched")
+    ap.add_argument("--fused-step", action="store_true",
+                    help="decode steps through thinK_append_decode (append + attention in one call, the attention "
+                         "launched as a programmatic dependent); decode.us_per_step is then the whole step")
     ap.add_argument("--lam", type=float, default=None, help="override the config's pruning ratio (c5 sweep)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

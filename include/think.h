@@ -236,6 +236,14 @@ thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, 
 thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
                                void* stream);
 
+/* One decode step in one call: thinK_append followed by thinK_decode_attn for the same layers (Sec. 3.3),
+ * same arguments and results.  The attention kernel is launched as a programmatic dependent of the append
+ * kernel: it starts streaming the pruned prefix while the append is still running and waits for it only
+ * where it first touches the tail, which takes the append and the launch gap off the step's critical path.
+ * bf16 caches; fp32 caches run the two launches back to back. */
+thinK_status thinK_append_decode(thinK_cache* c, const void* k_new, const void* v_new, const void* q, void* out,
+                                 int32_t layer0, int32_t nlayers, void* stream);
+
 /* Score + select without any caller- or library-side allocation.  (The paper has no counterpart:
  * this is a packaging variant of thinK_score_select, same kernel, same results.)
  *

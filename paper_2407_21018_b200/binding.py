@@ -61,6 +61,8 @@ EXPORTS = {
                                         C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_v_kept_bytes": (C.c_size_t, [C.c_void_p]),
     "thinK_append": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
+    "thinK_append_decode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                      C.c_void_p]),
     "thinK_decode_attn": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_score_select_static": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32), Tensor5, Tensor5, C.c_int32,
                                             C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -236,6 +238,17 @@ class ThinKCache:
             out = torch.empty_like(q)
         _check(lib.thinK_decode_attn(self.handle, q.data_ptr(), out.data_ptr(), layer0, nlayers, _stream_ptr(stream)),
                "thinK_decode_attn")
+        return out
+
+    def append_decode(self, k_new: torch.Tensor, v_new: torch.Tensor, q: torch.Tensor, out: Optional[torch.Tensor] = None,
+                      layer0=0, nlayers=None, stream=None):
+        """append + decode_attn in one call (the attention kernel overlaps the append)."""
+        nlayers = self.cfg.L - layer0 if nlayers is None else nlayers
+        assert k_new.is_contiguous() and v_new.is_contiguous() and q.is_contiguous()
+        if out is None:
+            out = torch.empty_like(q)
+        _check(lib.thinK_append_decode(self.handle, k_new.data_ptr(), v_new.data_ptr(), q.data_ptr(), out.data_ptr(),
+                                       layer0, nlayers, _stream_ptr(stream)), "thinK_append_decode")
         return out
 
     def reprune_tail(self, keep_recent: int, layer0=0, nlayers=None, stream=None):

@@ -176,6 +176,9 @@ __global__ void __launch_bounds__(128) k_reprune_bf16(const RepruneParams p) {
 // one row: the value chunk is copied as is, the key chunk is scattered into the channel-major tile.
 template <typename Tin>
 __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
+  // a kernel launched behind this one as a programmatic dependent may start now (it synchronises on this
+  // grid's completion itself before it reads what is written here); without such a launch this is a no-op
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   constexpr int E = sizeof(Tin);
   constexpr int CH = 16 / E;
   const int cpr = p.D / CH;

@@ -186,6 +186,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       i_left = min(p.seq_len[b] - p.R, je * kTileTokens) - j0 * kTileTokens;
     } else if (j0 - nthin < p.n_re) {
       // tail blocks that were re-pruned: keys thinned like the prefix, values still in the tail buffer
+      asm volatile("griddepcontrol.wait;" ::: "memory");   // the append ahead of this launch has written the tail
       const int jb = j0 - nthin, je = min(j1 - nthin, p.n_re);
       ntiles = je - jb;
       i_kstep = Tp * 32;
@@ -196,6 +197,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
       v0 = (const unsigned char*)p.tail_v + (unit_abs * p.cap + (int64_t)jb * kTileTokens) * D * 2;
       i_left = ntiles * kTileTokens;
     } else {
+      asm volatile("griddepcontrol.wait;" ::: "memory");   // the append ahead of this launch has written the tail
       const int jb = j0 - nthin, je = j1 - nthin;
       ntiles = je - jb;
       i_kstep = D * 32;
@@ -509,6 +511,21 @@ __global__ void __launch_bounds__(kWarps * 32, 1) k_decode_mma(const DecodeParam
 template <int D, int G>
 cudaError_t launch_mma(const DecodeParams& p, cudaStream_t s) {
   constexpr int smem = kSmemBytes + kWarps * (G * D * 2 + 128);
+  if (p.dependent_launch) {
+    // programmatic dependent launch: the grid may start while the append kernel ahead of it in the stream is
+    // still running; only workers that reach tail tiles wait for it (griddepcontrol.wait in the kernel)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.grid);
+    cfg.blockDim = dim3(kWarps * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return p.v_thin ? cudaLaunchKernelEx(&cfg, k_decode_mma<D, G, true>, p) : cudaLaunchKernelEx(&cfg, k_decode_mma<D, G, false>, p);
+  }
   if (p.v_thin) k_decode_mma<D, G, true><<<p.grid, kWarps * 32, smem, s>>>(p);
   else k_decode_mma<D, G, false><<<p.grid, kWarps * 32, smem, s>>>(p);
   return cudaGetLastError();

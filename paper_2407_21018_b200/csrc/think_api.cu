@@ -540,8 +540,8 @@ thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, 
   return THINK_OK;
 }
 
-thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
-                               void* stream) {
+static thinK_status decode_impl(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
+                                void* stream, bool dependent_launch) {
   if (!c || !q || !out) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out)) return THINK_ERR_INVALID_ARG;
@@ -579,8 +579,22 @@ thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t
   for (int b = 0; b < g.B; ++b)
     if (g.cum_thin[b + 1] - g.cum_thin[b] + p.n_tail_tiles < 1) return THINK_ERR_STATE;  // nothing to attend to
   p.grid = (int)(p.Ntot < (long long)c->decode_grid_max ? p.Ntot : (long long)c->decode_grid_max);
+  p.dependent_launch = dependent_launch && g.dtype == THINK_BF16;
   if (launch_decode(p, g.dtype, g.D, g.G, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
   return THINK_OK;
+}
+
+thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
+                               void* stream) {
+  return decode_impl(c, q, out, layer0, nlayers, stream, false);
+}
+
+thinK_status thinK_append_decode(thinK_cache* c, const void* k_new, const void* v_new, const void* q, void* out,
+                                 int32_t layer0, int32_t nlayers, void* stream) {
+  if (!c || !q || !out || !aligned16(q) || !aligned16(out)) return THINK_ERR_INVALID_ARG;   // nothing launched
+  thinK_status st = thinK_append(c, k_new, v_new, layer0, nlayers, stream);
+  if (st != THINK_OK) return st;
+  return decode_impl(c, q, out, layer0, nlayers, stream, true);
 }
 
 thinK_status thinK_reprune_tail(thinK_cache* c, int32_t keep_recent, int32_t layer0, int32_t nlayers, void* stream) {

@@ -147,6 +147,8 @@ struct DecodeParams {
   int layer0, nlayers;
   long long Ntot;           // tiles over all units of this call
   int grid;
+  int dependent_launch;     // host side: launch so that the kernel may start while the preceding kernel of the
+                            // stream (the append) is still running; it waits before its first read of the tail
 };
 
 // launchers (one per translation unit); return the launch status

@@ -254,6 +254,43 @@ def test_value_channel_pruning_state_and_support():
     assert e.value.status == tk.ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("name,lam_v", [("c2", 0.0), ("c4", 0.0), ("c2", 0.3), ("c1", 0.0)])
+def test_append_decode_in_one_call(name, lam_v):
+    """thinK_append_decode (attention launched as a programmatic dependent of the append) gives bit-identical
+    outputs and cache contents to thinK_append + thinK_decode_attn, step after step, and matches the oracle."""
+    base = wl.get_config(name)
+    w = wl.shrink(base, S=900, L=min(base.L, 2), B=min(base.B, 3), steps=70)
+    data = wl.make_prefill(w, device="cuda")
+    a, b = make_cache(w, w.steps, lam_v=lam_v), make_cache(w, w.steps, lam_v=lam_v)
+    for c in (a, b):
+        c.prefill(data["Q_obs"], data["K"], data["V"])
+    o = make_oracle(w, lam_v)
+    K64, V64, Q64 = to64(data["K"]), to64(data["V"]), to64(data["Q_obs"])
+    o.score_select(Q64, K64)
+    compare_selection(a.idx_tensor().cpu().numpy(), None, o, w.name)
+    if lam_v > 0:
+        o.score_select_v(Q64, K64, V64)
+        compare_selection(a.perm_v_tensor().cpu().numpy()[..., : o.T_v], None, o, w.name + " values", values=True)
+    o.compact(K64, V64)
+    for t in range(w.steps):
+        st = wl.make_step(w, t, device="cuda")
+        a.append(st["k_new"], st["v_new"])
+        out_a = a.decode_attn(st["q"])
+        out_b = b.append_decode(st["k_new"], st["v_new"], st["q"])
+        torch.cuda.synchronize()
+        assert torch.equal(out_a, out_b), f"step {t}: fused step differs from the two calls"
+        o.append(to64(st["k_new"]), to64(st["v_new"]))
+        if t % 23 == 0 or t == w.steps - 1:
+            assert_attn_close(to64(out_b), o.decode_attn(to64(st["q"])), w.dtype, f"{w.name} step {t}")
+    from paper_2407_21018_b200 import binding as tk
+    for (bb, l, h) in [(0, 0, 0), (w.B - 1, w.L - 1, w.N_kv - 1)]:
+        ka, va = tk.tail_logical(a, bb, l, h)
+        kb, vb = tk.tail_logical(b, bb, l, h)
+        assert torch.equal(ka, kb) and torch.equal(va, vb)
+    assert a.tail_len() == b.tail_len() == w.recent + w.steps
+    assert b.device_error() == 0
+
+
 @pytest.mark.parametrize("lam", [0.0, 0.25, 0.75])
 def test_lambda_sweep(lam):
     w = wl.shrink(wl.get_config("c5"), S=1000, L=1, steps=3, lam=lam)
