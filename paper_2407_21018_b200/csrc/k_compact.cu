@@ -74,6 +74,11 @@ __global__ void __launch_bounds__(128) k_compact(const CompactParams p) {
 template <bool TOK>
 __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
   extern __shared__ __align__(16) unsigned char smem[];
+  // Launched as a programmatic dependent of the kernel ahead of it (the score pass): the grid is scheduled
+  // while that kernel drains, waits here for its results, and only then lets its own dependent (the tail
+  // seed, which reads nothing this kernel writes) go.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int D = p.D, T = p.T, Tp = p.Tp;
   const int pitch = D * 2 + 16;
   unsigned char* s_in = smem;                                   // [64][pitch]
@@ -322,8 +327,17 @@ cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cud
   cudaError_t e;
   if (dtype == THINK_BF16) {
     smem = (size_t)kTileTokens * (p.D * 2 + 16) + ((p.Tp + 15) & ~15);
-    if (p.tok.rows) k_compact_bf16<true><<<grid, 128, smem, s>>>(p);
-    else k_compact_bf16<false><<<grid, 128, smem, s>>>(p);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return p.tok.rows ? cudaLaunchKernelEx(&cfg, k_compact_bf16<true>, p) : cudaLaunchKernelEx(&cfg, k_compact_bf16<false>, p);
   } else if (p.tok.rows) {
     e = cudaFuncSetAttribute(k_compact<float, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -342,12 +356,26 @@ cudaError_t launch_reprune(const RepruneParams& p, cudaStream_t s) {
   return cudaGetLastError();
 }
 
-cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s) {
+// `overlap_previous`: the kernel ahead in the stream writes nothing this launch reads or writes and has itself
+// waited for everything before it (the compaction kernel at prefill), so the two may run side by side.
+cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s, bool overlap_previous) {
   const int E = dtype == THINK_BF16 ? 2 : 4;
   const int64_t total = (int64_t)p.B * p.nlayers * p.N_kv * p.nrows * (p.D * E / 16);
   if (total <= 0) return cudaSuccess;
   int blocks = (int)((total + 255) / 256);
   if (blocks > kSMs * 16) blocks = kSMs * 16;
+  if (overlap_previous && dtype == THINK_BF16) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_tail_write<__nv_bfloat16>, p);
+  }
   if (dtype == THINK_BF16) k_tail_write<__nv_bfloat16><<<blocks, 256, 0, s>>>(p);
   else k_tail_write<float><<<blocks, 256, 0, s>>>(p);
   return cudaGetLastError();

@@ -43,6 +43,8 @@ __device__ __forceinline__ uint4 ldg16(const void* p) {
 
 template <typename Tin, bool L1, bool TOK>
 __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const ScoreParams p) {
+  // the compaction kernel behind this launch may be scheduled now; it waits for this grid before it reads idx
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   constexpr int CH = Chunk<Tin>::CH;
   constexpr bool kBf16 = sizeof(Tin) == 2;
   __shared__ double red[kScoreThreads * CH];   // reused: row-lane reduction, then scores

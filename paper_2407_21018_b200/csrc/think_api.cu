@@ -383,7 +383,8 @@ thinK_status seed_tail(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, const T
     t.tail_k = c->tail_k; t.tail_v = c->tail_v;
     t.B = g.B; t.L = g.L; t.N_kv = g.N_kv; t.D = g.D; t.R = g.R; t.cap = g.cap; t.tail_tiles_cap = g.tail_tiles_cap;
     t.layer0 = layer0; t.nlayers = nlayers; t.nrows = g.R; t.pos0 = 0;
-    if (launch_tail_write(t, g.dtype, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+    // with value pruning the kernel ahead is the value compaction, which does not let dependents go early
+    if (launch_tail_write(t, g.dtype, (cudaStream_t)stream, !g.vt) != cudaSuccess) return THINK_ERR_CUDA;
   }
   c->v = v_prefix;
   c->have_v = true;

@@ -155,7 +155,7 @@ struct DecodeParams {
 cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s);
 int score_ctas_per_sm(int dtype, int criterion);
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s);
-cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s);
+cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s, bool overlap_previous = false);
 cudaError_t launch_reprune(const RepruneParams& p, cudaStream_t s);
 cudaError_t launch_score_value(const ValueScoreParams& p, int threads, cudaStream_t s);
 cudaError_t score_value_setup(int D);
