@@ -333,6 +333,32 @@ def test_shapes(dtype, D, G):
     run_case(w)
 
 
+@pytest.mark.parametrize("D,G,lam_v", [(64, 8, 0.5), (64, 2, 0.3), (128, 8, 0.3), (128, 2, 0.6)])
+def test_value_channel_pruning_shapes(D, G, lam_v):
+    """Value-channel pruning on the other head shapes: D = 64 (mma.sync score kernel), group sizes 2 and 8
+    (S_obs = 16: 32 or 128 stacked window rows), ragged batch."""
+    w = wl.Workload("vshape", "bf16", 2, 2, 2 * G, 2, D, (300, 171), 16, 0.4, 3, 10000.0, (2, 10.0), 0x5EED + D + G)
+    data = wl.make_prefill(w, device="cpu")
+    cache = make_cache(w, w.steps, lam_v=lam_v)
+    cache.prefill(data["Q_obs"].cuda(), data["K"].cuda(), data["V"].cuda())
+    o = make_oracle(w, lam_v)
+    K64, V64, Q64 = to64(data["K"]), to64(data["V"]), to64(data["Q_obs"])
+    o.score_select(Q64, K64)
+    o.score_select_v(Q64, K64, V64)
+    compare_selection(cache.idx_tensor().cpu().numpy(), cache.scores_tensor().cpu().numpy(), o, w.name)
+    compare_selection(cache.perm_v_tensor().cpu().numpy()[..., : o.T_v], cache.scores_v_tensor().cpu().numpy(), o,
+                      w.name + " values", values=True)
+    o.compact(K64, V64)
+    compare_cache(cache, o, where=w.name)
+    for t in range(w.steps):
+        st = wl.make_step(w, t, device="cpu")
+        out = cache.append_decode(st["k_new"].cuda(), st["v_new"].cuda(), st["q"].cuda())
+        torch.cuda.synchronize()
+        o.append(to64(st["k_new"]), to64(st["v_new"]))
+        assert_attn_close(to64(out), o.decode_attn(to64(st["q"])), w.dtype, f"{w.name} step {t}")
+    assert cache.device_error() == 0
+
+
 @pytest.mark.parametrize("criterion", [1, 2])
 def test_magnitude_criteria(criterion):
     """Eq. 1 criteria (key l2 / l1 norms) through the same kernels."""
