@@ -294,8 +294,7 @@ def run_ours(args):
                 dq.copy_(s["q"], non_blocking=True)
                 dk.copy_(s["k_new"], non_blocking=True)
                 dv.copy_(s["v_new"], non_blocking=True)
-                cache.append(dk, dv)
-                cache.decode_attn(dq, out=out)
+                cache.append_decode(dk, dv, dq, out=out)
                 hout.copy_(out, non_blocking=True)
         e2e_pass()
         torch.cuda.synchronize()
