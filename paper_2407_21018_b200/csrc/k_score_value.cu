@@ -68,17 +68,18 @@ __device__ __forceinline__ void split_pair_packed(float x0, float x1, uint32_t& 
 
 // Ticket + finaliser shared by both kernels: the CTA that arrives last for the unit merges the splits
 // row by row (in split order), forms the column norms over all M rows in fp64 and ranks the channels.
-// `smem`: scratch of at least nsplit*M*4 + (kRowGroups + 1)*D*8 bytes, free to overwrite.
+// `smem`: scratch of at least nsplit*M*4 + (kRowGroups + 1)*D*8 bytes, free to overwrite; `s_last_slot`: one int of
+// shared memory outside that scratch; `arrivals`: token splits this CTA stands for.
 template <int D>
-__device__ void finish_unit(const ValueScoreParams& p, unsigned char* smem, int ucall, int b, int l, int h) {
-  __shared__ int s_last;
+__device__ void finish_unit(const ValueScoreParams& p, unsigned char* smem, int* s_last_slot, int ucall, int b, int l, int h,
+                            int arrivals = 1) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x;
   const size_t rec_floats = (size_t)p.MB * (2 + D);
   __threadfence();
   __syncthreads();
-  if (tid == 0) s_last = atomicAdd(p.counters + ucall, 1u) == (uint32_t)(p.nrb * p.nsplit - 1);
+  if (tid == 0) *s_last_slot = atomicAdd(p.counters + ucall, (uint32_t)arrivals) == (uint32_t)(p.nrb * p.nsplit - arrivals);
   __syncthreads();
-  if (!s_last) return;
+  if (!*s_last_slot) return;
   __threadfence();
 
   float* w = (float*)smem;                                   // [nsplit][M]: weight of a split's row / its denominator
@@ -288,7 +289,8 @@ __global__ void __launch_bounds__(256, 1) k_score_value(const ValueScoreParams p
       *(float2*)(ob + 8 * t) = make_float2(o[t][2], o[t][3]);
     }
   }
-  finish_unit<D>(p, smem, ucall, b, l, h);
+  __shared__ int s_last;
+  finish_unit<D>(p, smem, &s_last, ucall, b, l, h);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -582,7 +584,308 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
   if (warp == 0)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(tmem), "r"(kTcCols) : "memory");
   if (!ok_all) return;
-  finish_unit<D>(p, smem, ucall, b, l, h);
+  __shared__ int s_last_tc;
+  finish_unit<D>(p, smem, &s_last_tc, ucall, b, l, h);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Two software pipelines per CTA with their own MMA warps (one CTA per SM, 320 threads).
+// Measured on the kernel above: per 64-token tile a CTA spends ~1150 cycles in the softmax and ~1270 cycles in
+// the one thread that issues the 16 MMAs (the issue blocks while the tensor pipe executes them), one after the
+// other, because that thread also owns a softmax row.  Here the roles are split:
+//   * warpgroup w (128 threads, w = 0, 1) runs the softmax of pipeline w on its half of the CTA's token range;
+//   * warp 8 + w only issues pipeline w's MMAs; it is told by named barriers (arrive by the 128 softmax threads,
+//     sync by the 32 issuing lanes) when K(t+1) has landed and when P(t) and V(t) are in place;
+//   * K and V have two buffers each and S two sets of tensor-memory columns, so the first product of tile t+1
+//     and the copies of tiles t+1, t+2 run under the softmax of tile t, and the second product of tile t under
+//     the softmax of tile t+1 (whose weights wait in registers until the P buffers are free again).
+// Status: correct (same tests), but not faster than the kernel above on c2/c5 (321 vs 307 us, 8.5 vs 8.3 ms), so it
+// is not the default.  Measured per 64-token tile and pipeline: 3.8 K cycles, of which 1.8 K softmax arithmetic
+// and 0.9 K + 1.0 K in the MMA warp's two issue bursts at ~115 cycles per MMA whatever its N: the operands of
+// every MMA come from shared memory (176 KB per tile and pipeline), which is what paces the issue; and a CTA now
+// holds a whole SM, so 256 units leave 1.73 waves.
+// Only Q is shared by the two pipelines.  Waits on mbarriers stay bounded; a pipeline that times out raises the
+// error word, from then on meets its MMA warp at every barrier in step (so that nobody is left waiting and no
+// barrier receives two rounds of arrivals) and issues nothing more.
+// ---------------------------------------------------------------------------------------------
+constexpr int kT2Threads = 320;
+constexpr int kT2Pipe = 98304;                 // per pipeline: K x 2 | V x 2 | P hi | P lo
+constexpr int kT2K = 0, kT2V = 32768, kT2Phi = 65536, kT2Plo = 81920;
+constexpr int kT2Bars = 32768 + 2 * kT2Pipe;   // after Q and the two pipelines
+constexpr int kT2Bytes = kT2Bars + 64;
+constexpr int kT2Cols = 512;                   // per pipeline 256: S x 2 (64 each) | O (128)
+
+__device__ __forceinline__ bool wg_and(int id, bool x) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(r) : "r"((uint32_t)x), "r"(id) : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ bool wg_or(int id, bool x) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
+      : "=r"(r) : "r"((uint32_t)x), "r"(id) : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void bar_arrive160(int id) { asm volatile("bar.arrive %0, 160;" :: "r"(id) : "memory"); }
+__device__ __forceinline__ void bar_sync160(int id) { asm volatile("bar.sync %0, 160;" :: "r"(id) : "memory"); }
+
+__global__ void __launch_bounds__(kT2Threads, 1) k_score_value_tc2(const ValueScoreParams p) {
+  constexpr int D = 128;
+  // no static shared memory: the dynamic window then starts on the 1024-byte boundary the swizzled operands need
+  extern __shared__ __align__(1024) unsigned char smem_t2[];
+  unsigned char* const smem = smem_t2;
+  const uint32_t sb = smem_u32(smem);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const bool mma_warp = warp >= 8;
+  const int wg = mma_warp ? warp - 8 : tid >> 7;      // pipeline of this thread
+  const int wt = tid & 127;
+  const int id_wg = 1 + wg, id_qk = 3 + 2 * wg, id_pv = 4 + 2 * wg;
+  const int rb = blockIdx.y, ucall = blockIdx.z;
+  const int split = 2 * blockIdx.x + wg;              // p.nsplit = 2 * gridDim.x token splits per (unit, row block)
+  const int h = ucall % p.N_kv, bl = ucall / p.N_kv;
+  const int ll = bl % p.nlayers, b = bl / p.nlayers, l = p.layer0 + ll;
+  if ((sb & 1023u) != 0) {
+    if (tid == 0 && p.error) atomicOr(p.error, kErrSmemAlign);
+    return;
+  }
+  const int S_b = p.seq_len[b];
+  const int ntile_all = (S_b + kVTile - 1) / kVTile;
+  const int per = (ntile_all + p.nsplit - 1) / p.nsplit;
+  const int t0 = min(S_b, split * per * kVTile), t1 = min(S_b, (split + 1) * per * kVTile);
+  const int ntl = (t1 - t0 + kVTile - 1) / kVTile;
+  const uint32_t pipe = sb + 32768 + wg * kT2Pipe;
+  const uint32_t bar_s = sb + kT2Bars + wg * 16, bar_o = bar_s + 8;
+  volatile uint32_t* s_tmem = (volatile uint32_t*)(smem + kT2Bars + 32);
+  int* s_last = (int*)(smem + kT2Bars + 36);
+  volatile int* s_abort = (volatile int*)(smem + kT2Bars + 40) + wg;   // this pipeline has given up
+
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(sb + kT2Bars + 32), "r"(kT2Cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (!mma_warp && wt == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar_s) : "memory");
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar_o) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    *s_abort = 0;
+  }
+  auto swz = [](int r, int ck, int block_bytes) -> uint32_t {
+    return (uint32_t)((ck >> 3) * block_bytes + (r >> 3) * 1024 + (r & 7) * 128 + (((ck & 7) ^ (r & 7)) << 4));
+  };
+  const __nv_bfloat16* kg = (const __nv_bfloat16*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn;
+  const __nv_bfloat16* vg = (const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;
+  auto load_tile = [&](uint32_t dst, const __nv_bfloat16* g, int64_t stride, int t) {   // tile t of this pipeline's range
+    if (t < ntl) {
+      const int tok0 = t0 + t * kVTile;
+#pragma unroll
+      for (int i = 0; i < kVTile * 16 / 128; ++i) {
+        const int idx = wt + i * 128, r = idx >> 4, ck = idx & 15;
+        const bool ok = tok0 + r < t1;             // rows past the range are zero-filled
+        cp_async16_zfill(dst + swz(r, ck, 8192), g + (int64_t)(ok ? tok0 + r : t0) * stride + ck * 8, ok ? 16 : 0);
+      }
+    }
+    cp_commit();
+  };
+  if (!mma_warp) {
+    // query rows (shared by both pipelines): row r of the unit = query head h*G + r / S_obs, window row r % S_obs
+    const int r = rb * p.MB + wt;
+    const bool ok = r < p.M;
+    const __nv_bfloat16* q = (const __nv_bfloat16*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl +
+                             (int64_t)(ok ? r % p.S_obs : 0) * p.q.ss + (int64_t)(h * p.G + (ok ? r / p.S_obs : 0)) * p.q.sn;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) cp_async16_zfill(sb + swz(wt, wg * 8 + c, 16384), q + (wg * 8 + c) * 8, ok ? 16 : 0);
+    load_tile(pipe + kT2K, kg, p.k.ss, 0);           // group: Q (this thread's part) + K(0)
+    load_tile(pipe + kT2K + 16384, kg, p.k.ss, 1);   // group: K(1)
+    load_tile(pipe + kT2V, vg, p.v.ss, 0);           // group: V(0)
+    cp_wait<2>();                                    // Q + K(0)
+    fence_proxy_async();
+  }
+  tc_fence_before();
+  __syncthreads();                                   // Q is complete only when both warpgroups have copied their part
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem + (uint32_t)wg * 256;                   // this pipeline's columns
+  const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16);    // a warp reaches the 32 lanes of its rank mod 4
+  constexpr uint32_t kColS1 = 64, kColO = 128;
+  bool ok_all = true;
+
+  if (mma_warp) {
+    // ---------------- the pipeline's MMA warp: lane 0 issues, all lanes take part in the barriers
+    auto issue_qk = [&](int t) {                     // S buffer t & 1 = Q K(t)^T, keys in K buffer t & 1
+      const uint32_t kb = pipe + kT2K + (t & 1) * 16384;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks)
+        umma_bf16(tmem + (uint32_t)(t & 1) * kColS1, umma_desc(sb + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+                  umma_desc(kb + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), kIdescQK, ks > 0);
+      umma_commit(bar_s);
+    };
+    if (ntl > 0 && lane == 0) issue_qk(0);
+    for (int it = 0; it < ntl; ++it) {
+      if (it + 1 < ntl) {
+        bar_sync160(id_qk);                          // K(it + 1) has landed and S buffer (it + 1) & 1 has been read
+        tc_fence_after();
+        if (lane == 0 && !*s_abort) issue_qk(it + 1);
+      }
+      bar_sync160(id_pv);                            // P(it) is stored and V(it) has landed
+      tc_fence_after();
+      if (lane == 0 && !*s_abort) {
+        const uint32_t vbuf = pipe + kT2V + (it & 1) * 16384;
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16(tmem + kColO, umma_desc(pipe + kT2Phi + ks * 32, 16, 1024), umma_desc(vbuf + ks * 2048, 8192, 1024),
+                    kIdescPV, (it > 0 || ks > 0) ? 1u : 0u);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks)
+          umma_bf16(tmem + kColO, umma_desc(pipe + kT2Plo + ks * 32, 16, 1024), umma_desc(vbuf + ks * 2048, 8192, 1024),
+                    kIdescPV, 1u);
+        umma_commit(bar_o);
+      }
+    }
+  } else {
+    // ---------------- the pipeline's softmax warpgroup
+    const float scale = 1.4426950408889634f / sqrtf((float)D);
+    float m_used = -INFINITY, lsum = 0.f;
+    for (int it = 0; it < ntl; ++it) {
+      if (!ok_all) {                                 // given up: keep the MMA warp's barriers moving, in step with it
+        if (it + 1 < ntl) bar_sync160(id_qk);
+        bar_sync160(id_pv);
+        continue;
+      }
+      // ---- S(it) is ready
+      if (!wg_and(id_wg, mbar_wait(bar_s, it & 1))) {
+        ok_all = false; *s_abort = 1;
+        if (it + 1 < ntl) bar_sync160(id_qk);
+        bar_sync160(id_pv);
+        continue;
+      }
+      tc_fence_after();
+      if (it + 1 < ntl) {                            // the next tile's first product can go out at once
+        cp_wait<1>();                                // everything but the latest group, V(it): K(it + 1) has landed
+        fence_proxy_async();
+        tc_fence_before();
+        bar_arrive160(id_qk);
+      }
+      load_tile(pipe + kT2K + (it & 1) * 16384, kg, p.k.ss, it + 2);    // K buffer it & 1 is free: group K(it + 2)
+
+      // ---- this thread's row of S(it): masked past the range; running maximum in the exp2 domain
+      uint32_t sr[2][32];
+      const uint32_t tS = tlane + (uint32_t)(it & 1) * kColS1;
+      tmem_ld32(tS, sr[0]);
+      tmem_ld32(tS + 32, sr[1]);
+      tmem_wait_ld();
+      const int nvalid = min(kVTile, t1 - (t0 + it * kVTile));
+      if (nvalid < kVTile) {
+#pragma unroll
+        for (int j = 0; j < 64; ++j)
+          if (j >= nvalid) sr[j >> 5][j & 31] = 0xff800000u;   // -inf
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < 64; j += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(sr[j >> 5][j & 31]));
+        mx1 = fmaxf(mx1, __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]));
+        mx2 = fmaxf(mx2, __uint_as_float(sr[(j + 2) >> 5][(j + 2) & 31]));
+        mx3 = fmaxf(mx3, __uint_as_float(sr[(j + 3) >> 5][(j + 3) & 31]));
+      }
+      const float m_new = fmaxf(m_used, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale);   // scale > 0
+      // raising the maximum rescales O, which the second product of tile it - 1 may still be writing
+      bool pv_waited = it == 0;
+      const bool raise = m_new > m_used + 8.f;
+      if (wg_or(id_wg, raise)) {
+        if (!pv_waited) {
+          if (!wg_and(id_wg, mbar_wait(bar_o, (it - 1) & 1))) { ok_all = false; *s_abort = 1; bar_sync160(id_pv); continue; }
+          tc_fence_after();
+          pv_waited = true;
+        }
+        if (__any_sync(0xffffffffu, raise)) {
+          const float factor = ex2(m_used - m_new);
+          if (it > 0) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < D; c0 += 32) {
+              uint32_t o[32];
+              tmem_ld32(tlane + kColO + c0, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
+              tmem_st32(tlane + kColO + c0, o);
+            }
+            tmem_wait_st();
+          }
+          lsum *= factor;
+          m_used = m_new;
+        }
+      }
+      // ---- P = hi + lo in registers, while the tensor pipe works on S(it + 1) and O(it - 1)
+      const float neg_m = -m_used;
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t hi[32], lo[32];
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        const int j = 2 * e;
+        const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), scale, neg_m));
+        const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), scale, neg_m));
+        ls[e & 3] += p0 + p1;      // the denominator takes the weights before the hi + lo split (2^-17 apart)
+        split_pair_packed(p0, p1, hi[e], lo[e]);
+      }
+      lsum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      // ---- the second product of tile it - 1 is done: P buffers and value buffer (it + 1) & 1 are free
+      if (!pv_waited) {
+        if (!wg_and(id_wg, mbar_wait(bar_o, (it - 1) & 1))) { ok_all = false; *s_abort = 1; bar_sync160(id_pv); continue; }
+        tc_fence_after();
+      }
+      load_tile(pipe + kT2V + ((it + 1) & 1) * 16384, vg, p.v.ss, it + 1);   // group V(it + 1)
+      const uint32_t prow = (uint32_t)((wt >> 3) * 1024 + (wt & 7) * 128);
+#pragma unroll
+      for (int tc = 0; tc < 8; ++tc) {
+        const uint32_t off = prow + ((uint32_t)(tc ^ (wt & 7)) << 4);
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(pipe + kT2Phi + off), "r"(hi[4 * tc]), "r"(hi[4 * tc + 1]), "r"(hi[4 * tc + 2]), "r"(hi[4 * tc + 3]) : "memory");
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(pipe + kT2Plo + off), "r"(lo[4 * tc]), "r"(lo[4 * tc + 1]), "r"(lo[4 * tc + 2]), "r"(lo[4 * tc + 3]) : "memory");
+      }
+      cp_wait<2>();                                  // V(it) has landed; K(it + 2) and V(it + 1) may be in flight
+      fence_proxy_async();
+      tc_fence_before();
+      bar_arrive160(id_pv);
+    }
+    if (ok_all && ntl > 0) {                         // the last second product
+      if (!wg_and(id_wg, mbar_wait(bar_o, (ntl - 1) & 1))) ok_all = false;
+      tc_fence_after();
+    }
+    cp_wait<0>();
+
+    // ---- partial state of this thread's row, same record as the other kernels
+    if (ok_all) {
+      const size_t rec_floats = (size_t)p.MB * (2 + D);
+      float* rec = p.partials + ((size_t)(ucall * p.nrb + rb) * p.nsplit + split) * rec_floats;
+      rec[wt] = m_used;
+      rec[p.MB + wt] = lsum;
+      float4* orow = (float4*)(rec + 2 * p.MB + (size_t)wt * D);
+#pragma unroll 1
+      for (int c0 = 0; c0 < D; c0 += 32) {
+        uint32_t o[32];
+        if (ntl > 0) {
+          tmem_ld32(tlane + kColO + c0, o);
+          tmem_wait_ld();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] = 0u;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          orow[c0 / 4 + j] = make_float4(__uint_as_float(o[4 * j]), __uint_as_float(o[4 * j + 1]), __uint_as_float(o[4 * j + 2]),
+                                         __uint_as_float(o[4 * j + 3]));
+      }
+    } else if (wt == 0 && p.error) {
+      atomicOr(p.error, kErrWaitTimeout);
+    }
+  }
+  tc_fence_before();
+  const bool both = __syncthreads_and(ok_all);       // both pipelines are through
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(*s_tmem), "r"(kT2Cols) : "memory");
+  if (!both) return;
+  finish_unit<D>(p, smem, s_last, ucall, b, l, h, 2);
 }
 
 constexpr int smem_bytes(int D) { return kVStages * 2 * kVTile * D * 2; }
@@ -595,6 +898,8 @@ cudaError_t score_value_setup(int D) {
   if (D == 128) {
     cudaError_t e = cudaFuncSetAttribute(k_score_value_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcBytes + 1024);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_score_value_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, kT2Bytes);
+    if (e != cudaSuccess) return e;
   }
   if (D == 128) return cudaFuncSetAttribute(k_score_value<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128));
   if (D == 64) return cudaFuncSetAttribute(k_score_value<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64));
@@ -604,6 +909,10 @@ cudaError_t score_value_setup(int D) {
 // threads = 32 * (MB / 16): one warp per 16 query rows of the row block
 cudaError_t launch_score_value(const ValueScoreParams& p, int threads, cudaStream_t s) {
   dim3 grid(p.nsplit, p.nrb, p.B * p.nlayers * p.N_kv);
+  if (p.use_tcgen05 == 2 && p.D == 128 && p.MB == 128 && p.nsplit % 2 == 0) {
+    k_score_value_tc2<<<dim3(p.nsplit / 2, p.nrb, p.B * p.nlayers * p.N_kv), kT2Threads, kT2Bytes, s>>>(p);
+    return cudaGetLastError();
+  }
   if (p.use_tcgen05 && p.D == 128 && p.MB == 128) {
     k_score_value_tc<<<grid, kTcThreads, kTcBytes + 1024, s>>>(p);
     return cudaGetLastError();

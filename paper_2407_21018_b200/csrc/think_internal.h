@@ -30,6 +30,7 @@ struct TokenMap {
 };
 constexpr uint32_t kErrTokenRange = 1u;   // device error word: a token index was out of range
 constexpr uint32_t kErrWaitTimeout = 2u;  // device error word: a bounded wait on an mbarrier ran out
+constexpr uint32_t kErrSmemAlign = 4u;    // device error word: dynamic shared memory not on a 1024-byte boundary
 
 struct ScoreParams {
   TokenMap tok;
@@ -91,7 +92,7 @@ struct ValueScoreParams {    // App. D: Score_v = column norms of the window's a
   int M;                    // G * S_obs query rows per unit
   int MB;                   // rows per row block (multiple of 16, <= 128)
   int nrb, nsplit;
-  int use_tcgen05;          // D = 128 and MB = 128: tcgen05.mma kernel instead of the mma.sync one
+  int use_tcgen05;          // D = 128 and MB = 128: 0 mma.sync kernel, 1 tcgen05 (one pipeline per CTA), 2 two pipelines per CTA
   uint32_t* error;          // device error word
 };
 
