@@ -298,10 +298,10 @@ __global__ void __launch_bounds__(256, 1) k_score_value(const ValueScoreParams p
 // memory), for D = 128 and blocks of 128 query rows.  A CTA of 128 threads owns (token split, row
 // block, unit); thread t owns query row t = tensor-memory lane t.
 //   per tile of 64 tokens:   S = Q K^T      one thread issues 8 MMAs (M128 N64 K16), S in TMEM columns [0, 64) or [64, 128)
-//                            softmax        every thread reads its row of S, writes P = hi + lo as bf16 rows
-//                            O += P V       one thread issues 4 + 4 MMAs (M128 N128 K16), O in columns [128, 256)
-// Operands sit in shared memory in the canonical 128-byte-swizzled layouts (rows of 128 bytes, 16-byte
-// chunk index XOR row%8, 1024-byte groups of 8 rows): Q, K and P K-major, V MN-major -- which is exactly
+//                            softmax        every thread reads its row of S and writes P = hi + lo (bf16) back over it
+//                            O += P V       one thread issues 4 + 4 MMAs (M128 N128 K16, A = P from tensor memory), O in columns [128, 256)
+// Q, K and V sit in shared memory in the canonical 128-byte-swizzled layouts (rows of 128 bytes, 16-byte
+// chunk index XOR row%8, 1024-byte groups of 8 rows): Q and K K-major, V MN-major -- which is exactly
 // V's natural [token][channel] order, so no transpose is needed.  The running maximum is only raised when it
 // grows by more than 8 (in the exp2 domain): O in tensor memory is then rescaled, otherwise the stale
 // maximum stays and numerator and denominator simply carry the same bounded factor.
@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(256, 1) k_score_value(const ValueScoreParams p
 // time-out the CTA raises the error word, releases its tensor memory and leaves without a ticket.
 // ---------------------------------------------------------------------------------------------
 constexpr int kTcThreads = 128;
-constexpr int kTcQ = 0, kTcK = 32768, kTcV = 49152, kTcPhi = 65536, kTcPlo = 81920, kTcBytes = 98304;
+constexpr int kTcQ = 0, kTcK = 32768, kTcV = 49152, kTcBytes = 65536;   // Q | K tile | V tile
 constexpr int kTcCols = 256;              // allocated tensor-memory columns (power of two): 2 x S 64 + O 128
 constexpr uint32_t kTcColS1 = 64, kTcColO = 128;   // S buffers at columns 0 and 64, O at 128
 // instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128; N and the majorness of B differ
@@ -331,6 +331,16 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t"
       "}\n"
       :: "r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
+}
+// the same with the A operand in tensor memory (row = lane, K elements packed two per 32-bit column)
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t"
+      "}\n"
+      :: "r"(tmem_d), "r"(tmem_a), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" :: "r"(bar) : "memory");
@@ -508,25 +518,23 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
       lsum *= factor;
       m_used = m_new;
     }
-    // ---- P = hi + lo, written as rows of the two A operands
-    const uint32_t prow = (uint32_t)((tid >> 3) * 1024 + (tid & 7) * 128);
+    // ---- P = hi + lo goes back into tensor memory, over the S columns it was computed from: as the A operand
+    // of the second product it is read from there (a row per lane, two bf16 per 32-bit column), so the weights
+    // never pass through shared memory and the MMA reads only V from it
     const float neg_m = -m_used;
     float ls[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t hi[32], lo[32];
 #pragma unroll
-    for (int tc = 0; tc < 8; ++tc) {
-      uint32_t hi[4], lo[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int j = 8 * tc + 2 * e;
-        const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), scale, neg_m));
-        const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), scale, neg_m));
-        ls[e] += p0 + p1;          // the denominator takes the weights before the hi + lo split (2^-17 apart)
-        split_pair_packed(p0, p1, hi[e], lo[e]);
-      }
-      const uint32_t off = prow + ((uint32_t)(tc ^ (tid & 7)) << 4);
-      asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(sb + kTcPhi + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
-      asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(sb + kTcPlo + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+    for (int e = 0; e < 32; ++e) {
+      const int j = 2 * e;
+      const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), scale, neg_m));
+      const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), scale, neg_m));
+      ls[e & 3] += p0 + p1;        // the denominator takes the weights before the hi + lo split (2^-17 apart)
+      split_pair_packed(p0, p1, hi[e], lo[e]);
     }
+    tmem_st32(tS, hi);             // columns [0, 32) of this S buffer: P hi, tokens 2c, 2c + 1 in column c
+    tmem_st32(tS + 32, lo);        // columns [32, 64): P lo
+    tmem_wait_st();
     lsum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
     cp_wait<0>();                 // V(it) and K(it + 1) have landed
     fence_proxy_async();
@@ -534,14 +542,14 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
     __syncthreads();
     if (tid == 0) {
       tc_fence_after();
+      const uint32_t tP = tmem + (uint32_t)(it & 1) * kTcColS1;      // 16 tokens = 8 columns per MMA
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks)
-        umma_bf16(tmem + kTcColO, umma_desc(sb + kTcPhi + ks * 32, 16, 1024), umma_desc(sb + kTcV + ks * 2048, 8192, 1024),
-                  kIdescPV, (it > 0 || ks > 0) ? 1u : 0u);
+        umma_bf16_ts(tmem + kTcColO, tP + ks * 8, umma_desc(sb + kTcV + ks * 2048, 8192, 1024), kIdescPV,
+                     (it > 0 || ks > 0) ? 1u : 0u);
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks)
-        umma_bf16(tmem + kTcColO, umma_desc(sb + kTcPlo + ks * 32, 16, 1024), umma_desc(sb + kTcV + ks * 2048, 8192, 1024),
-                  kIdescPV, 1u);
+        umma_bf16_ts(tmem + kTcColO, tP + 32 + ks * 8, umma_desc(sb + kTcV + ks * 2048, 8192, 1024), kIdescPV, 1u);
       umma_commit(bar_o);
       // the next tile's first product goes to the other S buffer right behind it: its round trip hides
       // behind this tile's second product instead of adding to it
