@@ -456,12 +456,15 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
   const float scale = 1.4426950408889634f / sqrtf((float)D);
   float m_used = -INFINITY, lsum = 0.f;
   bool ok_all = true;
+  // operand descriptors are built once: inside the loops a k-step only adds a constant to the address field
+  // (16-byte units)
+  const uint64_t dQ = umma_desc(sb + kTcQ, 16, 1024), dK = umma_desc(sb + kTcK, 16, 1024), dV = umma_desc(sb + kTcV, 8192, 1024);
   // first product of tile `t` into S buffer t & 1 (issued by one thread)
   auto issue_qk = [&](int t) {
 #pragma unroll
     for (int ks = 0; ks < 8; ++ks)
-      umma_bf16(tmem + (uint32_t)(t & 1) * kTcColS1, umma_desc(sb + kTcQ + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                umma_desc(sb + kTcK + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), kIdescQK, ks > 0);
+      umma_bf16(tmem + (uint32_t)(t & 1) * kTcColS1, dQ + (uint64_t)((ks >> 2) * 1024 + (ks & 3) * 2),
+                dK + (uint64_t)((ks >> 2) * 512 + (ks & 3) * 2), kIdescQK, ks > 0);
     umma_commit(bar_s);
   };
   if (ntl > 0) {
@@ -545,11 +548,10 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
       const uint32_t tP = tmem + (uint32_t)(it & 1) * kTcColS1;      // 16 tokens = 8 columns per MMA
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks)
-        umma_bf16_ts(tmem + kTcColO, tP + ks * 8, umma_desc(sb + kTcV + ks * 2048, 8192, 1024), kIdescPV,
-                     (it > 0 || ks > 0) ? 1u : 0u);
+        umma_bf16_ts(tmem + kTcColO, tP + ks * 8, dV + (uint64_t)(ks * 128), kIdescPV, (it > 0 || ks > 0) ? 1u : 0u);
 #pragma unroll
       for (int ks = 0; ks < 4; ++ks)
-        umma_bf16_ts(tmem + kTcColO, tP + 32 + ks * 8, umma_desc(sb + kTcV + ks * 2048, 8192, 1024), kIdescPV, 1u);
+        umma_bf16_ts(tmem + kTcColO, tP + 32 + ks * 8, dV + (uint64_t)(ks * 128), kIdescPV, 1u);
       umma_commit(bar_o);
       // the next tile's first product goes to the other S buffer right behind it: its round trip hides
       // behind this tile's second product instead of adding to it
@@ -597,31 +599,30 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
 }
 
 // ---------------------------------------------------------------------------------------------
-// Two software pipelines per CTA with their own MMA warps (one CTA per SM, 320 threads).
-// Measured on the kernel above: per 64-token tile a CTA spends ~1150 cycles in the softmax and ~1270 cycles in
-// the one thread that issues the 16 MMAs (the issue blocks while the tensor pipe executes them), one after the
-// other, because that thread also owns a softmax row.  Here the roles are split:
-//   * warpgroup w (128 threads, w = 0, 1) runs the softmax of pipeline w on its half of the CTA's token range;
-//   * warp 8 + w only issues pipeline w's MMAs; it is told by named barriers (arrive by the 128 softmax threads,
-//     sync by the 32 issuing lanes) when K(t+1) has landed and when P(t) and V(t) are in place;
+// The same kernel with the roles split (160 threads, two CTAs per SM).  Selectable, tested, NOT the default: it
+// is slower than the kernel above (c2: 385 vs 301 us).  What the measurements say: in the kernel above a CTA
+// spends per 64-token tile ~1150 cycles in the softmax and ~1270 cycles in the one thread that issues the 16 MMAs,
+// one after the other, because that thread also owns a softmax row; the 16 MMAs themselves need only ~800 cycles
+// of the tensor pipe.  With the roles split as below the MMA warp waits ~1700 cycles per tile for the softmax
+// warps, whose per-tile work (tensor-memory load, 64 exponentials and hi + lo conversions, the 16 cp.async of the
+// next K and V tiles, the stores of P) is then the critical path; the next steps are a copy warp (bulk tensor
+// copies instead of per-thread cp.async) and two threads per row.  Structure:
+//   * warps 0-3 (128 threads, one query row each) run the softmax;
+//   * warp 4 only issues MMAs; named barriers (arrive by the 128 softmax threads, sync by the 32 issuing lanes)
+//     tell it when K(t+1) has landed and when P(t) and V(t) are in place;
 //   * K and V have two buffers each and S two sets of tensor-memory columns, so the first product of tile t+1
 //     and the copies of tiles t+1, t+2 run under the softmax of tile t, and the second product of tile t under
-//     the softmax of tile t+1 (whose weights wait in registers until the P buffers are free again).
-// Status: correct (same tests), but not faster than the kernel above on c2/c5 (321 vs 307 us, 8.5 vs 8.3 ms), so it
-// is not the default.  Measured per 64-token tile and pipeline: 3.8 K cycles, of which 1.8 K softmax arithmetic
-// and 0.9 K + 1.0 K in the MMA warp's two issue bursts at ~115 cycles per MMA whatever its N: the operands of
-// every MMA come from shared memory (176 KB per tile and pipeline), which is what paces the issue; and a CTA now
-// holds a whole SM, so 256 units leave 1.73 waves.
-// Only Q is shared by the two pipelines.  Waits on mbarriers stay bounded; a pipeline that times out raises the
-// error word, from then on meets its MMA warp at every barrier in step (so that nobody is left waiting and no
-// barrier receives two rounds of arrivals) and issues nothing more.
+//     the softmax of tile t+1 (whose weights wait in registers until the product of tile t-1 has released O
+//     and the S columns they go to).
+// Waits on mbarriers stay bounded; a CTA that times out raises the error word, from then on meets its MMA warp
+// at every barrier in step (so that nobody is left waiting and no barrier receives two rounds of arrivals) and
+// issues nothing more.
 // ---------------------------------------------------------------------------------------------
-constexpr int kT2Threads = 320;
-constexpr int kT2Pipe = 98304;                 // per pipeline: K x 2 | V x 2 | P hi | P lo
-constexpr int kT2K = 0, kT2V = 32768, kT2Phi = 65536, kT2Plo = 81920;
-constexpr int kT2Bars = 32768 + 2 * kT2Pipe;   // after Q and the two pipelines
+constexpr int kT2Threads = 160;
+constexpr int kT2K = 0, kT2V = 32768;          // after Q: K x 2 | V x 2
+constexpr int kT2Bars = 32768 + 65536;
 constexpr int kT2Bytes = kT2Bars + 64;
-constexpr int kT2Cols = 512;                   // per pipeline 256: S x 2 (64 each) | O (128)
+constexpr int kT2Cols = 256;                   // S x 2 (64 each) | O (128)
 
 __device__ __forceinline__ bool wg_and(int id, bool x) {
   uint32_t r;
@@ -647,12 +648,10 @@ __global__ void __launch_bounds__(kT2Threads, 1) k_score_value_tc2(const ValueSc
   unsigned char* const smem = smem_t2;
   const uint32_t sb = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool mma_warp = warp >= 8;
-  const int wg = mma_warp ? warp - 8 : tid >> 7;      // pipeline of this thread
+  const bool mma_warp = warp == 4;
   const int wt = tid & 127;
-  const int id_wg = 1 + wg, id_qk = 3 + 2 * wg, id_pv = 4 + 2 * wg;
-  const int rb = blockIdx.y, ucall = blockIdx.z;
-  const int split = 2 * blockIdx.x + wg;              // p.nsplit = 2 * gridDim.x token splits per (unit, row block)
+  constexpr int id_wg = 1, id_qk = 2, id_pv = 3;
+  const int split = blockIdx.x, rb = blockIdx.y, ucall = blockIdx.z;
   const int h = ucall % p.N_kv, bl = ucall / p.N_kv;
   const int ll = bl % p.nlayers, b = bl / p.nlayers, l = p.layer0 + ll;
   if ((sb & 1023u) != 0) {
@@ -664,11 +663,11 @@ __global__ void __launch_bounds__(kT2Threads, 1) k_score_value_tc2(const ValueSc
   const int per = (ntile_all + p.nsplit - 1) / p.nsplit;
   const int t0 = min(S_b, split * per * kVTile), t1 = min(S_b, (split + 1) * per * kVTile);
   const int ntl = (t1 - t0 + kVTile - 1) / kVTile;
-  const uint32_t pipe = sb + 32768 + wg * kT2Pipe;
-  const uint32_t bar_s = sb + kT2Bars + wg * 16, bar_o = bar_s + 8;
+  const uint32_t pipe = sb + 32768;
+  const uint32_t bar_s = sb + kT2Bars, bar_o = bar_s + 8;
   volatile uint32_t* s_tmem = (volatile uint32_t*)(smem + kT2Bars + 32);
   int* s_last = (int*)(smem + kT2Bars + 36);
-  volatile int* s_abort = (volatile int*)(smem + kT2Bars + 40) + wg;   // this pipeline has given up
+  volatile int* s_abort = (volatile int*)(smem + kT2Bars + 40);       // the softmax side has given up
 
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(sb + kT2Bars + 32), "r"(kT2Cols) : "memory");
@@ -698,35 +697,37 @@ __global__ void __launch_bounds__(kT2Threads, 1) k_score_value_tc2(const ValueSc
     cp_commit();
   };
   if (!mma_warp) {
-    // query rows (shared by both pipelines): row r of the unit = query head h*G + r / S_obs, window row r % S_obs
+    // query row of this thread: row r of the unit = query head h*G + r / S_obs, window row r % S_obs
     const int r = rb * p.MB + wt;
     const bool ok = r < p.M;
     const __nv_bfloat16* q = (const __nv_bfloat16*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl +
                              (int64_t)(ok ? r % p.S_obs : 0) * p.q.ss + (int64_t)(h * p.G + (ok ? r / p.S_obs : 0)) * p.q.sn;
 #pragma unroll
-    for (int c = 0; c < 8; ++c) cp_async16_zfill(sb + swz(wt, wg * 8 + c, 16384), q + (wg * 8 + c) * 8, ok ? 16 : 0);
-    load_tile(pipe + kT2K, kg, p.k.ss, 0);           // group: Q (this thread's part) + K(0)
+    for (int c = 0; c < 16; ++c) cp_async16_zfill(sb + swz(wt, c, 16384), q + c * 8, ok ? 16 : 0);
+    load_tile(pipe + kT2K, kg, p.k.ss, 0);           // group: Q (this thread's row) + K(0)
     load_tile(pipe + kT2K + 16384, kg, p.k.ss, 1);   // group: K(1)
     load_tile(pipe + kT2V, vg, p.v.ss, 0);           // group: V(0)
     cp_wait<2>();                                    // Q + K(0)
     fence_proxy_async();
   }
   tc_fence_before();
-  __syncthreads();                                   // Q is complete only when both warpgroups have copied their part
+  __syncthreads();                                   // Q and K(0) are complete, the tensor-memory address is published
   tc_fence_after();
-  const uint32_t tmem = *s_tmem + (uint32_t)wg * 256;                   // this pipeline's columns
+  const uint32_t tmem = *s_tmem;
   const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16);    // a warp reaches the 32 lanes of its rank mod 4
   constexpr uint32_t kColS1 = 64, kColO = 128;
   bool ok_all = true;
 
   if (mma_warp) {
-    // ---------------- the pipeline's MMA warp: lane 0 issues, all lanes take part in the barriers
+    // ---------------- the MMA warp: lane 0 issues, all lanes take part in the barriers
+    // descriptors once; a k-step or the other buffer only adds a constant to the address field (16-byte units)
+    const uint64_t dQ = umma_desc(sb, 16, 1024), dK = umma_desc(pipe + kT2K, 16, 1024), dV = umma_desc(pipe + kT2V, 8192, 1024);
     auto issue_qk = [&](int t) {                     // S buffer t & 1 = Q K(t)^T, keys in K buffer t & 1
-      const uint32_t kb = pipe + kT2K + (t & 1) * 16384;
+      const uint64_t dKt = dK + (uint64_t)((t & 1) * 1024);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks)
-        umma_bf16(tmem + (uint32_t)(t & 1) * kColS1, umma_desc(sb + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-                  umma_desc(kb + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), kIdescQK, ks > 0);
+        umma_bf16(tmem + (uint32_t)(t & 1) * kColS1, dQ + (uint64_t)((ks >> 2) * 1024 + (ks & 3) * 2),
+                  dKt + (uint64_t)((ks >> 2) * 512 + (ks & 3) * 2), kIdescQK, ks > 0);
       umma_commit(bar_s);
     };
     if (ntl > 0 && lane == 0) issue_qk(0);
@@ -739,20 +740,19 @@ __global__ void __launch_bounds__(kT2Threads, 1) k_score_value_tc2(const ValueSc
       bar_sync160(id_pv);                            // P(it) is stored and V(it) has landed
       tc_fence_after();
       if (lane == 0 && !*s_abort) {
-        const uint32_t vbuf = pipe + kT2V + (it & 1) * 16384;
+        const uint64_t dVt = dV + (uint64_t)((it & 1) * 1024);
+        const uint32_t tP = tmem + (uint32_t)(it & 1) * kColS1;          // P(it) lies over S(it): 8 columns per MMA
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          umma_bf16(tmem + kColO, umma_desc(pipe + kT2Phi + ks * 32, 16, 1024), umma_desc(vbuf + ks * 2048, 8192, 1024),
-                    kIdescPV, (it > 0 || ks > 0) ? 1u : 0u);
+          umma_bf16_ts(tmem + kColO, tP + ks * 8, dVt + (uint64_t)(ks * 128), kIdescPV, (it > 0 || ks > 0) ? 1u : 0u);
 #pragma unroll
         for (int ks = 0; ks < 4; ++ks)
-          umma_bf16(tmem + kColO, umma_desc(pipe + kT2Plo + ks * 32, 16, 1024), umma_desc(vbuf + ks * 2048, 8192, 1024),
-                    kIdescPV, 1u);
+          umma_bf16_ts(tmem + kColO, tP + 32 + ks * 8, dVt + (uint64_t)(ks * 128), kIdescPV, 1u);
         umma_commit(bar_o);
       }
     }
   } else {
-    // ---------------- the pipeline's softmax warpgroup
+    // ---------------- the softmax warps
     const float scale = 1.4426950408889634f / sqrtf((float)D);
     float m_used = -INFINITY, lsum = 0.f;
     for (int it = 0; it < ntl; ++it) {
@@ -838,19 +838,15 @@ __global__ void __launch_bounds__(kT2Threads, 1) k_score_value_tc2(const ValueSc
         split_pair_packed(p0, p1, hi[e], lo[e]);
       }
       lsum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      // ---- the second product of tile it - 1 is done: P buffers and value buffer (it + 1) & 1 are free
+      // ---- the second product of tile it - 1 is done: value buffer (it + 1) & 1 is free
       if (!pv_waited) {
         if (!wg_and(id_wg, mbar_wait(bar_o, (it - 1) & 1))) { ok_all = false; *s_abort = 1; bar_sync160(id_pv); continue; }
         tc_fence_after();
       }
       load_tile(pipe + kT2V + ((it + 1) & 1) * 16384, vg, p.v.ss, it + 1);   // group V(it + 1)
-      const uint32_t prow = (uint32_t)((wt >> 3) * 1024 + (wt & 7) * 128);
-#pragma unroll
-      for (int tc = 0; tc < 8; ++tc) {
-        const uint32_t off = prow + ((uint32_t)(tc ^ (wt & 7)) << 4);
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(pipe + kT2Phi + off), "r"(hi[4 * tc]), "r"(hi[4 * tc + 1]), "r"(hi[4 * tc + 2]), "r"(hi[4 * tc + 3]) : "memory");
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" :: "r"(pipe + kT2Plo + off), "r"(lo[4 * tc]), "r"(lo[4 * tc + 1]), "r"(lo[4 * tc + 2]), "r"(lo[4 * tc + 3]) : "memory");
-      }
+      tmem_st32(tS, hi);             // P(it) over S(it): hi in columns [0, 32), lo in [32, 64), two tokens per column
+      tmem_st32(tS + 32, lo);
+      tmem_wait_st();
       cp_wait<2>();                                  // V(it) has landed; K(it + 2) and V(it + 1) may be in flight
       fence_proxy_async();
       tc_fence_before();
@@ -889,11 +885,11 @@ __global__ void __launch_bounds__(kT2Threads, 1) k_score_value_tc2(const ValueSc
     }
   }
   tc_fence_before();
-  const bool both = __syncthreads_and(ok_all);       // both pipelines are through
+  const bool both = __syncthreads_and(ok_all);       // softmax warps and MMA warp are through
   if (warp == 0)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(*s_tmem), "r"(kT2Cols) : "memory");
   if (!both) return;
-  finish_unit<D>(p, smem, s_last, ucall, b, l, h, 2);
+  finish_unit<D>(p, smem, s_last, ucall, b, l, h);
 }
 
 constexpr int smem_bytes(int D) { return kVStages * 2 * kVTile * D * 2; }
@@ -917,8 +913,8 @@ cudaError_t score_value_setup(int D) {
 // threads = 32 * (MB / 16): one warp per 16 query rows of the row block
 cudaError_t launch_score_value(const ValueScoreParams& p, int threads, cudaStream_t s) {
   dim3 grid(p.nsplit, p.nrb, p.B * p.nlayers * p.N_kv);
-  if (p.use_tcgen05 == 2 && p.D == 128 && p.MB == 128 && p.nsplit % 2 == 0) {
-    k_score_value_tc2<<<dim3(p.nsplit / 2, p.nrb, p.B * p.nlayers * p.N_kv), kT2Threads, kT2Bytes, s>>>(p);
+  if (p.use_tcgen05 == 2 && p.D == 128 && p.MB == 128) {
+    k_score_value_tc2<<<grid, kT2Threads, kT2Bytes, s>>>(p);
     return cudaGetLastError();
   }
   if (p.use_tcgen05 && p.D == 128 && p.MB == 128) {

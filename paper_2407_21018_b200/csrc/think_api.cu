@@ -226,8 +226,8 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
   c->k_thin = k_thin; c->tail_k = tail_k; c->tail_v = tail_v; c->idx = idx; c->scores = scores;
   c->v_thin = c->perm_v = c->scores_v = nullptr;
   {
-    // which value-score kernel serves 128-row blocks at D = 128: "mma_sync", "tcgen05_2" (two pipelines per CTA
-    // with their own MMA warps; not faster so far) or, by default, the tcgen05 kernel with one pipeline per CTA
+    // which value-score kernel serves 128-row blocks at D = 128: "mma_sync", "tcgen05_2" (softmax warps + a
+    // separate MMA warp, double-buffered K/V) or, by default, the tcgen05 kernel whose threads share the roles
     const char* e = getenv("THINK_VALUE_SCORE");
     c->value_score_tcgen05 = e && strcmp(e, "mma_sync") == 0 ? 0 : (e && strcmp(e, "tcgen05_2") == 0 ? 2 : 1);
   }
@@ -452,20 +452,14 @@ thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_te
   if (max_split < 1) max_split = 1;
   // the split that wastes least of the last wave of CTAs (ties: the smaller split, less to merge)
   const bool tc = p.use_tcgen05 && g.D == 128 && g.MB == 128;
-  if (tc && p.use_tcgen05 == 2 && max_split < 2) p.use_tcgen05 = 1;     // too short for two pipelines per CTA
-  const bool two = tc && p.use_tcgen05 == 2;                             // a CTA then covers two token splits
-  const int resident = c->num_sms * (two ? 1 : tc ? 2 : (g.MB >= 128 ? 1 : 2));
-  int nsplit = two ? 2 : 1;
+  const int resident = c->num_sms * (tc ? 2 : (g.MB >= 128 ? 1 : 2));
+  int nsplit = 1;
   double best = 0.0;
-  for (int s = nsplit; s <= max_split; s += two ? 2 : 1) {
-    const long long recs = (long long)per_layer * per_launch * s, ctas = two ? recs / 2 : recs;
-    if (recs > g.value_slots) break;
+  for (int s = 1; s <= max_split; ++s) {
+    const long long ctas = (long long)per_layer * per_launch * s;
+    if (ctas > g.value_slots) break;
     const double waves = (double)ctas / resident, eff = waves / ceil(waves);
     if (eff > best + 1e-9) { best = eff; nsplit = s; }
-  }
-  if ((long long)per_layer * per_launch * nsplit > g.value_slots) {      // even the smallest split overflows the records
-    per_launch = g.value_slots / (per_layer * nsplit);
-    if (per_launch < 1) { per_launch = 1; nsplit = 1; p.use_tcgen05 = p.use_tcgen05 ? 1 : 0; }
   }
   p.nsplit = nsplit;
   for (int l0 = layer0; l0 < layer0 + nlayers; l0 += per_launch) {
