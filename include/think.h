@@ -170,7 +170,11 @@ thinK_status thinK_attach_value_cache(thinK_cache* c, void* v_thin, void* perm_v
  * go to the lower channel.  Both products run on tensor cores in bf16 with fp32 accumulation, the
  * softmax weights as a bf16 pair hi + lo; column norms in fp64.  Against an fp64 evaluation the scores
  * carry a relative error of about 1e-5, so two channels whose scores are closer than that may swap.
- * Writes perm_v (kept channels ascending, then the rest ascending).  `v` as for thinK_compact. */
+ * Writes perm_v (kept channels ascending, then the rest ascending).  `v` as for thinK_compact.
+ * Kernels: blocks of 128 stacked window rows at D = 128 run on tcgen05.mma with accumulators in tensor memory,
+ * everything else on mma.sync; the environment variable THINK_VALUE_SCORE (read by thinK_create) = "mma_sync" or
+ * "tcgen05_2" selects the mma.sync kernel or the variant with a separate MMA warp instead (same results within the
+ * tolerance above; for testing and measurement). */
 thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v,
                                    int32_t layer0, int32_t nlayers, void* stream);
 
