@@ -216,11 +216,17 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
     unsigned char* tile = (unsigned char*)p.tail_k + (unit * p.tail_tiles_cap + u / kTileTokens) * (int64_t)p.D * kTileTokens * E;
     const Tin* kk = (const Tin*)&kv;
     const int uu = u % kTileTokens;
+    if (E == 2) {
+      // channels 2q, 2q + 1 of a token are neighbours in the fragment order: one 4-byte store per pair
+      const uint32_t* kw = (const uint32_t*)&kv;
 #pragma unroll
-    for (int j = 0; j < CH; ++j) {
-      int c = ck * CH + j;
-      if (E == 2) *(Tin*)(tile + frag_elem_byte(p.D, c, uu)) = kk[j];
-      else *(Tin*)(tile + c * kTileTokens * E + tile_swz_bytes(c, uu, E)) = kk[j];
+      for (int q = 0; q < 4; ++q) *(uint32_t*)(tile + frag_elem_byte(p.D, ck * 8 + 2 * q, uu)) = kw[q];
+    } else {
+#pragma unroll
+      for (int j = 0; j < CH; ++j) {
+        int c = ck * CH + j;
+        *(Tin*)(tile + c * kTileTokens * E + tile_swz_bytes(c, uu, E)) = kk[j];
+      }
     }
   }
 }
