@@ -386,10 +386,10 @@ def oracle_sample(w: wl.Workload, budget_s: float = 20.0):
         nbytes = prefill_bytes(ws, T) + sum(decode_bytes(ws, T, t) for t in range(steps)) + steps * append_bytes(ws)
         return t2 - t0, t1 - t0, t2 - t1, nbytes, ws
 
-    dt, _, _, _, _ = run(1, 1, 1)
-    scale = max(1.0, budget_s / max(dt, 1e-3))
-    L = int(max(1, min(w.L, scale ** 0.5)))
-    steps = int(max(1, min(w.steps, scale / L)))
+    run(1, 1, 1)                                     # warm-up of the numeric library's threads
+    _, pre1, dec1, _, _ = run(1, 1, 1)               # one layer, one decode step: cost of either phase per layer
+    steps = int(max(1, min(w.steps, 16)))
+    L = int(max(1, min(w.L, budget_s / max(pre1 + steps * dec1, 1e-3))))
     dt, dt_pre, dt_dec, nbytes, ws = run(L, 1, steps)
     return {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
             "sample": f"{ws.name}: B=1 of {w.B}, L={L} of {w.L}, S={ws.seq_lens[0]}, {steps} decode steps; "
