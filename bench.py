@@ -315,6 +315,7 @@ def run_ours(args):
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu = oracle_sample(w, budget_s=args.cpu_budget)
+        cpu.pop("sizing", None)
 
     if rank == 0:
         line = {
@@ -355,7 +356,7 @@ def run_ours(args):
 
 
 # --------------------------------------------------------------------------- the oracle arm
-def oracle_sample(w: wl.Workload, budget_s: float = 20.0):
+def oracle_sample(w: wl.Workload, budget_s: float = 20.0, sizing=None):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload: a few layers of
     the same prompts and a few decode steps, sized from a short probe so that it ends in about
     `budget_s` seconds.  Reported in the benchmark's unit (algorithmic bytes / wall time)."""
@@ -386,15 +387,20 @@ def oracle_sample(w: wl.Workload, budget_s: float = 20.0):
         nbytes = prefill_bytes(ws, T) + sum(decode_bytes(ws, T, t) for t in range(steps)) + steps * append_bytes(ws)
         return t2 - t0, t1 - t0, t2 - t1, nbytes, ws
 
-    run(1, 1, 1)                                     # warm-up of the numeric library's threads
-    _, pre1, dec1, _, _ = run(1, 1, 1)               # one layer, one decode step: cost of either phase per layer
-    steps = int(max(1, min(w.steps, 16)))
-    L = int(max(1, min(w.L, budget_s / max(pre1 + steps * dec1, 1e-3))))
+    if sizing is None:
+        run(1, 1, 1)                                 # warm-up of the numeric library's threads
+        _, pre1, dec1, _, _ = run(1, 1, 1)           # one layer, one decode step: cost of either phase per layer
+        steps = int(max(1, min(w.steps, 16)))
+        if budget_s < 4 * (pre1 + steps * dec1):     # small budgets: fewer decode steps before fewer layers
+            steps = int(max(1, min(steps, (budget_s / 2 - pre1) / max(dec1, 1e-6))))
+        L = int(max(1, min(w.L, budget_s / max(pre1 + steps * dec1, 1e-3))))
+    else:
+        L, steps = sizing
     dt, dt_pre, dt_dec, nbytes, ws = run(L, 1, steps)
     return {"value": nbytes / dt / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
             "sample": f"{ws.name}: B=1 of {w.B}, L={L} of {w.L}, S={ws.seq_lens[0]}, {steps} decode steps; "
                       f"prefill {dt_pre:.2f} s, decode {dt_dec / steps * 1e3:.1f} ms/step",
-            "seconds": dt}
+            "seconds": dt, "sizing": (L, steps)}
 
 
 def run_reference(args):
@@ -404,9 +410,12 @@ def run_reference(args):
     w = wl.get_config(args.config)
     vals = []
     last = None
-    per = max(2.0, min(60.0, 120.0 / max(1, args.steps + args.warmup)))
+    # the whole run is held to about two minutes: one probe sizes the sample, every step then times that sample
+    per = max(0.5, min(60.0, 120.0 / max(1, args.steps + args.warmup)))
+    sizing = None
     for i in range(args.warmup + args.steps):
-        last = oracle_sample(w, budget_s=per)
+        last = oracle_sample(w, budget_s=per, sizing=sizing)
+        sizing = last["sizing"]
         if i >= args.warmup:
             vals.append(last)
     v = sum(x["value"] for x in vals) / len(vals)
