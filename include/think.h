@@ -21,8 +21,9 @@
  *    return without synchronising.  Calls on one handle must be stream-ordered
  *    with respect to each other.
  *  - Errors are return codes.  Arguments are validated on the host before any
- *    launch; an invalid call launches nothing.  Inputs are assumed finite
- *    (NaN/Inf in K or Q leaves the selection unspecified).
+ *    launch; an invalid call launches nothing.  Inputs are assumed finite:
+ *    NaN/Inf in K or Q sets a bit of the device error word and leaves the
+ *    choice among the affected channels unspecified (never an out-of-range write).
  *  - Element type (`dtype`): bf16 or fp32 for K, V, Q, q, k_new, v_new and out.
  */
 #ifndef THINK_H_
@@ -53,6 +54,13 @@ typedef enum {
   THINK_SCORE_KEY_L1 = 2        /* Sec. 3.1, Eq. 1 with p = 1: ||K[:, j]||_1                    */
 } thinK_criterion;
 
+/* Kernel behind the value-channel score of App. D (thinK_score_select_kv). */
+typedef enum {
+  THINK_VALUE_SCORE_AUTO = 0,     /* tcgen05.mma with accumulators in tensor memory where the shape allows it
+                                     (blocks of 128 stacked window rows, D = 128), mma.sync elsewhere */
+  THINK_VALUE_SCORE_MMA_SYNC = 1  /* the mma.sync kernel everywhere (same results within the stated tolerance) */
+} thinK_value_score_kernel;
+
 typedef struct {
   int32_t B;              /* batch entries */
   int32_t L;              /* layers held by this cache */
@@ -65,7 +73,7 @@ typedef struct {
   int32_t max_new_tokens; /* decode steps the unpruned tail can take */
   int32_t dtype;          /* thinK_dtype */
   int32_t criterion;      /* thinK_criterion */
-  int32_t reserved;       /* 0 */
+  int32_t value_score_kernel; /* thinK_value_score_kernel; only read when lambda_v > 0 */
   double lambda;          /* pruning ratio, 0 <= lambda < 1 */
   double lambda_v;        /* pruning ratio of the value channels (App. D); 0 = values untouched (the default path) */
 } thinK_config;
@@ -136,10 +144,13 @@ thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens,
 
 /* Builds the host-side handle and writes the small device tables (lengths,
  * tile offsets, zeroed counters) into `workspace` with synchronous copies.
- * The buffers must be at least as large as thinK_cache_bytes reported and stay
- * valid until thinK_destroy.  `scores` may be NULL (scores are then not kept). */
-thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void* k_thin, void* tail_k,
-                          void* tail_v, void* idx, void* scores, void* workspace, thinK_cache** out);
+ * `sizes` (host) states the bytes the caller actually allocated for each buffer
+ * (v_thin and perm_v: for the later thinK_attach_value_cache); a buffer smaller
+ * than thinK_cache_bytes reports for this configuration is refused with
+ * THINK_ERR_CAPACITY before anything is written.  The buffers stay valid until
+ * thinK_destroy.  `scores` may be NULL (scores are then not kept). */
+thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, const thinK_sizes* sizes, void* k_thin,
+                          void* tail_k, void* tail_v, void* idx, void* scores, void* workspace, thinK_cache** out);
 
 /* Prefill, Sec. 3.2: channel scores and I = Top_T(Score, T) for layers
  * [layer0, layer0 + nlayers) of every (b, h).
@@ -172,9 +183,10 @@ thinK_status thinK_attach_value_cache(thinK_cache* c, void* v_thin, void* perm_v
  * carry a relative error of about 1e-5, so two channels whose scores are closer than that may swap.
  * Writes perm_v (kept channels ascending, then the rest ascending).  `v` as for thinK_compact.
  * Kernels: blocks of 128 stacked window rows at D = 128 run on tcgen05.mma with accumulators in tensor memory,
- * everything else on mma.sync; the environment variable THINK_VALUE_SCORE (read by thinK_create) = "mma_sync" or
- * "tcgen05_2" selects the mma.sync kernel or the variant with a separate MMA warp instead (same results within the
- * tolerance above; for testing and measurement). */
+ * everything else on mma.sync; cfg.value_score_kernel = THINK_VALUE_SCORE_MMA_SYNC keeps the mma.sync kernel
+ * everywhere (same results within the tolerance above).
+ * The tcgen05 kernel bounds its waits: if one runs out, the device error word gets bit 2 (see
+ * thinK_device_error) and the scores of that call are unspecified; the next call starts clean. */
 thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v,
                                    int32_t layer0, int32_t nlayers, void* stream);
 
@@ -182,7 +194,9 @@ thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_te
  * the idx thinK_score_select stored: K_T[t][c] = K[t][idx[c]] for t < S_p, and
  * the last S_recent rows of K and V copied unpruned to the tail.  After this
  * call K may be released by the caller; V rows [0, S_p) of `v` stay BORROWED:
- * thinK_decode_attn reads them in place on every step.
+ * thinK_decode_attn reads them in place on every step.  One view serves all
+ * layers: a call with a different `v` starts a new prompt, i.e. the layers
+ * outside its range count as not compacted until they are compacted again.
  * With lambda_v > 0 (after thinK_score_select_kv) the prefix values are thinned too:
  * V_T[t][c] = V[t][perm_v[c]], c < T_v, written to v_thin; the recent rows keep all D channels
  * (declared reading: App. D gives the criterion only; the split mirrors the keys').  `v` is then
@@ -263,9 +277,11 @@ thinK_status thinK_append_decode(thinK_cache* c, const void* k_new, const void* 
  *   idx:    device out, uint8 [B, L, N_kv, T]; rows of the given layers are written.
  *   scores: device out, fp64 [B, L, N_kv, D], or NULL.
  *
- * Limit: lengths + counters + 2 * B * nlayers * (N_kv*D) * 8 bytes per token split must fit in
- * 8 MiB.  The call lowers its token split to fit; if even one split does not fit it launches nothing
- * and returns THINK_ERR_CAPACITY -- pass fewer layers per call.
+ * Limit: lengths + counters + 2 * B * nlayers * C * 8 bytes per token split must fit in 8 MiB, where
+ * C = N_kv*D when a token's keys are at most 4096 bytes, else N_kv*D rounded up to a whole number of
+ * 4096-byte column blocks (2048 bf16 or 1024 fp32 columns each).  The call lowers its token split to
+ * fit; if even one split does not fit it launches nothing and returns THINK_ERR_CAPACITY -- pass
+ * fewer layers per call.
  * The first call on a device looks up the array's device address (once per device; make that first
  * call outside of any stream capture).  No cudaMalloc/cudaFree is called, here or later.
  * All calls share the one array, which still holds the previous call's contents: the call rewrites
@@ -291,7 +307,10 @@ int32_t thinK_repruned_len(const thinK_cache* c, int32_t layer);
 /* Tokens in the tail buffers of `layer` (S_recent + appended; re-pruned ones included), or -1. */
 int32_t thinK_tail_len(const thinK_cache* c, int32_t layer);
 
-/* Reads the device-side error word (0 = none) with a synchronous copy. */
+/* Reads the device-side error word (0 = none) with a synchronous copy.  Bits: 1 a kept-token index of
+ * thinK_prefill_evicted was out of range; 2 a bounded wait inside a kernel ran out; 4 a kernel found its
+ * shared memory misaligned; 8 a channel score was NaN or infinite (non-finite K or Q: exactly T channels
+ * are still selected, NaN scores ranking lowest). */
 thinK_status thinK_device_error(thinK_cache* c, int32_t* out_code);
 
 thinK_status thinK_destroy(thinK_cache* c);

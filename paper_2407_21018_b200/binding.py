@@ -14,7 +14,7 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.environ.get("THINK_LIB") or os.path.join(_HERE, "libthink.so")   # THINK_LIB: alternative build
+LIB_PATH = os.path.join(_HERE, "libthink.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -26,6 +26,8 @@ lib = C.CDLL(LIB_PATH)
 THINK_OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_STATE, ERR_CAPACITY, ERR_CUDA = range(6)
 BF16, F32 = 0, 1
 SCORE_QUERY_DRIVEN, SCORE_KEY_L2, SCORE_KEY_L1 = 0, 1, 2
+VALUE_SCORE_AUTO, VALUE_SCORE_MMA_SYNC = 0, 1
+ERR_BIT_TOKEN_RANGE, ERR_BIT_WAIT_TIMEOUT, ERR_BIT_SMEM_ALIGN, ERR_BIT_NON_FINITE = 1, 2, 4, 8
 TILE_TOKENS = 64
 
 
@@ -33,7 +35,7 @@ class Config(C.Structure):
     _fields_ = [("B", C.c_int32), ("L", C.c_int32), ("N_q", C.c_int32), ("N_kv", C.c_int32), ("D", C.c_int32),
                 ("S_max", C.c_int32), ("S_obs", C.c_int32), ("S_recent", C.c_int32),
                 ("max_new_tokens", C.c_int32), ("dtype", C.c_int32), ("criterion", C.c_int32),
-                ("reserved", C.c_int32), ("lam", C.c_double), ("lam_v", C.c_double)]
+                ("value_score_kernel", C.c_int32), ("lam", C.c_double), ("lam_v", C.c_double)]
 
 
 class Tensor5(C.Structure):
@@ -51,7 +53,8 @@ EXPORTS = {
     "thinK_T": (C.c_int32, [C.c_double, C.c_int32]),
     "thinK_status_string": (C.c_char_p, [C.c_int]),
     "thinK_cache_bytes": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32), C.POINTER(Sizes)]),
-    "thinK_create": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32)] + [C.c_void_p] * 6 + [C.POINTER(C.c_void_p)]),
+    "thinK_create": (C.c_int, [C.POINTER(Config), C.POINTER(C.c_int32), C.POINTER(Sizes)] + [C.c_void_p] * 6 +
+                     [C.POINTER(C.c_void_p)]),
     "thinK_score_select": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_compact": (C.c_int, [C.c_void_p, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
     "thinK_prefill": (C.c_int, [C.c_void_p, Tensor5, Tensor5, Tensor5, C.c_int32, C.c_int32, C.c_void_p]),
@@ -110,9 +113,10 @@ def tensor5(t: Optional[torch.Tensor]) -> Tensor5:
 
 
 def make_config(B, L, N_q, N_kv, D, S_max, S_obs, S_recent, max_new_tokens, lam, dtype, criterion=SCORE_QUERY_DRIVEN,
-                lam_v=0.0):
+                lam_v=0.0, value_score_kernel=VALUE_SCORE_AUTO):
     return Config(B, L, N_q, N_kv, D, S_max, S_obs, S_recent, max_new_tokens,
-                  dtype if isinstance(dtype, int) else _dtype_code(dtype), criterion, 0, float(lam), float(lam_v))
+                  dtype if isinstance(dtype, int) else _dtype_code(dtype), criterion, value_score_kernel, float(lam),
+                  float(lam_v))
 
 
 def thinK_cache_bytes(cfg: Config, seq_lens: Sequence[int]) -> Sizes:
@@ -161,8 +165,13 @@ class ThinKCache:
         self._v = None
         arr = (C.c_int32 * len(self.seq_lens))(*self.seq_lens)
         h = C.c_void_p()
+        # what was actually allocated, for the library's own size check
+        have = Sizes(self.k_thin.numel(), self.tail_k.numel(), self.tail_v.numel(), self.idx.numel(),
+                     self.scores.numel() if self.scores is not None else 0, self.workspace.numel(), 0, 0,
+                     max(int(self.sizes.v_thin), 256) if cfg.lam_v > 0 else 0,
+                     max(int(self.sizes.perm_v), 256) if cfg.lam_v > 0 else 0)
         with torch.cuda.device(self.device):
-            _check(lib.thinK_create(C.byref(cfg), arr, self.k_thin.data_ptr(), self.tail_k.data_ptr(),
+            _check(lib.thinK_create(C.byref(cfg), arr, C.byref(have), self.k_thin.data_ptr(), self.tail_k.data_ptr(),
                                     self.tail_v.data_ptr(), self.idx.data_ptr(),
                                     self.scores.data_ptr() if self.scores is not None else None,
                                     self.workspace.data_ptr(), C.byref(h)), "thinK_create")

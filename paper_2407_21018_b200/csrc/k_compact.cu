@@ -229,6 +229,10 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
       }
     }
   }
+  // When this grid was launched as a programmatic dependent (the tail seed beside the compaction kernel) it must
+  // not complete before the grid ahead of it: the next kernel in the stream waits for THIS grid only.  Without
+  // such a launch the instruction returns at once.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // Value-channel pruning (paper App. D): V_T[t][c] = V[t][perm_v[c]] for c < T_v, rows of Tvp elements

@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
   const int warp = tid >> 5, lane = tid & 31;
   for (int hh = warp; hh < heads; hh += kScoreThreads / 32) {
     const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h_first + hh;
-    select_head(red + hh * p.D, p.D, p.T, p.idx + unit * p.T, lane, false);
+    select_head(red + hh * p.D, p.D, p.T, p.idx + unit * p.T, lane, false, p.error);
     if (p.scores)
       for (int j = lane; j < p.D; j += 32) p.scores[unit * p.D + j] = red[hh * p.D + j];
   }

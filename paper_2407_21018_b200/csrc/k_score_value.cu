@@ -131,7 +131,7 @@ __device__ void finish_unit(const ValueScoreParams& p, unsigned char* smem, int*
   __syncthreads();
   const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
   if (warp == 0) {
-    select_head(sc, D, p.Tv, p.perm_v + unit * D, lane, true);
+    select_head(sc, D, p.Tv, p.perm_v + unit * D, lane, true, p.error);
     if (p.scores_v)
       for (int j = lane; j < D; j += 32) p.scores_v[unit * D + j] = sc[j];
   }
@@ -598,300 +598,6 @@ __global__ void __launch_bounds__(kTcThreads, 2) k_score_value_tc(const ValueSco
   finish_unit<D>(p, smem, &s_last_tc, ucall, b, l, h);
 }
 
-// ---------------------------------------------------------------------------------------------
-// The same kernel with the roles split (160 threads, two CTAs per SM).  Selectable, tested, NOT the default: it
-// is slower than the kernel above (c2: 385 vs 301 us).  What the measurements say: in the kernel above a CTA
-// spends per 64-token tile ~1150 cycles in the softmax and ~1270 cycles in the one thread that issues the 16 MMAs,
-// one after the other, because that thread also owns a softmax row; the 16 MMAs themselves need only ~800 cycles
-// of the tensor pipe.  With the roles split as below the MMA warp waits ~1700 cycles per tile for the softmax
-// warps, whose per-tile work (tensor-memory load, 64 exponentials and hi + lo conversions, the 16 cp.async of the
-// next K and V tiles, the stores of P) is then the critical path; the next steps are a copy warp (bulk tensor
-// copies instead of per-thread cp.async) and two threads per row.  Structure:
-//   * warps 0-3 (128 threads, one query row each) run the softmax;
-//   * warp 4 only issues MMAs; named barriers (arrive by the 128 softmax threads, sync by the 32 issuing lanes)
-//     tell it when K(t+1) has landed and when P(t) and V(t) are in place;
-//   * K and V have two buffers each and S two sets of tensor-memory columns, so the first product of tile t+1
-//     and the copies of tiles t+1, t+2 run under the softmax of tile t, and the second product of tile t under
-//     the softmax of tile t+1 (whose weights wait in registers until the product of tile t-1 has released O
-//     and the S columns they go to).
-// Waits on mbarriers stay bounded; a CTA that times out raises the error word, from then on meets its MMA warp
-// at every barrier in step (so that nobody is left waiting and no barrier receives two rounds of arrivals) and
-// issues nothing more.
-// ---------------------------------------------------------------------------------------------
-constexpr int kT2Threads = 160;
-constexpr int kT2K = 0, kT2V = 32768;          // after Q: K x 2 | V x 2
-constexpr int kT2Bars = 32768 + 65536;
-constexpr int kT2Bytes = kT2Bars + 64;
-constexpr int kT2Cols = 256;                   // S x 2 (64 each) | O (128)
-
-__device__ __forceinline__ bool wg_and(int id, bool x) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-      : "=r"(r) : "r"((uint32_t)x), "r"(id) : "memory");
-  return r != 0;
-}
-__device__ __forceinline__ bool wg_or(int id, bool x) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred p, %2, 128, q;\n\tselp.u32 %0, 1, 0, p;\n\t}\n"
-      : "=r"(r) : "r"((uint32_t)x), "r"(id) : "memory");
-  return r != 0;
-}
-__device__ __forceinline__ void bar_arrive160(int id) { asm volatile("bar.arrive %0, 160;" :: "r"(id) : "memory"); }
-__device__ __forceinline__ void bar_sync160(int id) { asm volatile("bar.sync %0, 160;" :: "r"(id) : "memory"); }
-
-__global__ void __launch_bounds__(kT2Threads, 1) k_score_value_tc2(const ValueScoreParams p) {
-  constexpr int D = 128;
-  // no static shared memory: the dynamic window then starts on the 1024-byte boundary the swizzled operands need
-  extern __shared__ __align__(1024) unsigned char smem_t2[];
-  unsigned char* const smem = smem_t2;
-  const uint32_t sb = smem_u32(smem);
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const bool mma_warp = warp == 4;
-  const int wt = tid & 127;
-  constexpr int id_wg = 1, id_qk = 2, id_pv = 3;
-  const int split = blockIdx.x, rb = blockIdx.y, ucall = blockIdx.z;
-  const int h = ucall % p.N_kv, bl = ucall / p.N_kv;
-  const int ll = bl % p.nlayers, b = bl / p.nlayers, l = p.layer0 + ll;
-  if ((sb & 1023u) != 0) {
-    if (tid == 0 && p.error) atomicOr(p.error, kErrSmemAlign);
-    return;
-  }
-  const int S_b = p.seq_len[b];
-  const int ntile_all = (S_b + kVTile - 1) / kVTile;
-  const int per = (ntile_all + p.nsplit - 1) / p.nsplit;
-  const int t0 = min(S_b, split * per * kVTile), t1 = min(S_b, (split + 1) * per * kVTile);
-  const int ntl = (t1 - t0 + kVTile - 1) / kVTile;
-  const uint32_t pipe = sb + 32768;
-  const uint32_t bar_s = sb + kT2Bars, bar_o = bar_s + 8;
-  volatile uint32_t* s_tmem = (volatile uint32_t*)(smem + kT2Bars + 32);
-  int* s_last = (int*)(smem + kT2Bars + 36);
-  volatile int* s_abort = (volatile int*)(smem + kT2Bars + 40);       // the softmax side has given up
-
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" :: "r"(sb + kT2Bars + 32), "r"(kT2Cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  if (!mma_warp && wt == 0) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar_s) : "memory");
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(bar_o) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    *s_abort = 0;
-  }
-  auto swz = [](int r, int ck, int block_bytes) -> uint32_t {
-    return (uint32_t)((ck >> 3) * block_bytes + (r >> 3) * 1024 + (r & 7) * 128 + (((ck & 7) ^ (r & 7)) << 4));
-  };
-  const __nv_bfloat16* kg = (const __nv_bfloat16*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn;
-  const __nv_bfloat16* vg = (const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;
-  auto load_tile = [&](uint32_t dst, const __nv_bfloat16* g, int64_t stride, int t) {   // tile t of this pipeline's range
-    if (t < ntl) {
-      const int tok0 = t0 + t * kVTile;
-#pragma unroll
-      for (int i = 0; i < kVTile * 16 / 128; ++i) {
-        const int idx = wt + i * 128, r = idx >> 4, ck = idx & 15;
-        const bool ok = tok0 + r < t1;             // rows past the range are zero-filled
-        cp_async16_zfill(dst + swz(r, ck, 8192), g + (int64_t)(ok ? tok0 + r : t0) * stride + ck * 8, ok ? 16 : 0);
-      }
-    }
-    cp_commit();
-  };
-  if (!mma_warp) {
-    // query row of this thread: row r of the unit = query head h*G + r / S_obs, window row r % S_obs
-    const int r = rb * p.MB + wt;
-    const bool ok = r < p.M;
-    const __nv_bfloat16* q = (const __nv_bfloat16*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl +
-                             (int64_t)(ok ? r % p.S_obs : 0) * p.q.ss + (int64_t)(h * p.G + (ok ? r / p.S_obs : 0)) * p.q.sn;
-#pragma unroll
-    for (int c = 0; c < 16; ++c) cp_async16_zfill(sb + swz(wt, c, 16384), q + c * 8, ok ? 16 : 0);
-    load_tile(pipe + kT2K, kg, p.k.ss, 0);           // group: Q (this thread's row) + K(0)
-    load_tile(pipe + kT2K + 16384, kg, p.k.ss, 1);   // group: K(1)
-    load_tile(pipe + kT2V, vg, p.v.ss, 0);           // group: V(0)
-    cp_wait<2>();                                    // Q + K(0)
-    fence_proxy_async();
-  }
-  tc_fence_before();
-  __syncthreads();                                   // Q and K(0) are complete, the tensor-memory address is published
-  tc_fence_after();
-  const uint32_t tmem = *s_tmem;
-  const uint32_t tlane = tmem + ((uint32_t)((warp & 3) * 32) << 16);    // a warp reaches the 32 lanes of its rank mod 4
-  constexpr uint32_t kColS1 = 64, kColO = 128;
-  bool ok_all = true;
-
-  if (mma_warp) {
-    // ---------------- the MMA warp: lane 0 issues, all lanes take part in the barriers
-    // descriptors once; a k-step or the other buffer only adds a constant to the address field (16-byte units)
-    const uint64_t dQ = umma_desc(sb, 16, 1024), dK = umma_desc(pipe + kT2K, 16, 1024), dV = umma_desc(pipe + kT2V, 8192, 1024);
-    auto issue_qk = [&](int t) {                     // S buffer t & 1 = Q K(t)^T, keys in K buffer t & 1
-      const uint64_t dKt = dK + (uint64_t)((t & 1) * 1024);
-#pragma unroll
-      for (int ks = 0; ks < 8; ++ks)
-        umma_bf16(tmem + (uint32_t)(t & 1) * kColS1, dQ + (uint64_t)((ks >> 2) * 1024 + (ks & 3) * 2),
-                  dKt + (uint64_t)((ks >> 2) * 512 + (ks & 3) * 2), kIdescQK, ks > 0);
-      umma_commit(bar_s);
-    };
-    if (ntl > 0 && lane == 0) issue_qk(0);
-    for (int it = 0; it < ntl; ++it) {
-      if (it + 1 < ntl) {
-        bar_sync160(id_qk);                          // K(it + 1) has landed and S buffer (it + 1) & 1 has been read
-        tc_fence_after();
-        if (lane == 0 && !*s_abort) issue_qk(it + 1);
-      }
-      bar_sync160(id_pv);                            // P(it) is stored and V(it) has landed
-      tc_fence_after();
-      if (lane == 0 && !*s_abort) {
-        const uint64_t dVt = dV + (uint64_t)((it & 1) * 1024);
-        const uint32_t tP = tmem + (uint32_t)(it & 1) * kColS1;          // P(it) lies over S(it): 8 columns per MMA
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          umma_bf16_ts(tmem + kColO, tP + ks * 8, dVt + (uint64_t)(ks * 128), kIdescPV, (it > 0 || ks > 0) ? 1u : 0u);
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          umma_bf16_ts(tmem + kColO, tP + 32 + ks * 8, dVt + (uint64_t)(ks * 128), kIdescPV, 1u);
-        umma_commit(bar_o);
-      }
-    }
-  } else {
-    // ---------------- the softmax warps
-    const float scale = 1.4426950408889634f / sqrtf((float)D);
-    float m_used = -INFINITY, lsum = 0.f;
-    for (int it = 0; it < ntl; ++it) {
-      if (!ok_all) {                                 // given up: keep the MMA warp's barriers moving, in step with it
-        if (it + 1 < ntl) bar_sync160(id_qk);
-        bar_sync160(id_pv);
-        continue;
-      }
-      // ---- S(it) is ready
-      if (!wg_and(id_wg, mbar_wait(bar_s, it & 1))) {
-        ok_all = false; *s_abort = 1;
-        if (it + 1 < ntl) bar_sync160(id_qk);
-        bar_sync160(id_pv);
-        continue;
-      }
-      tc_fence_after();
-      if (it + 1 < ntl) {                            // the next tile's first product can go out at once
-        cp_wait<1>();                                // everything but the latest group, V(it): K(it + 1) has landed
-        fence_proxy_async();
-        tc_fence_before();
-        bar_arrive160(id_qk);
-      }
-      load_tile(pipe + kT2K + (it & 1) * 16384, kg, p.k.ss, it + 2);    // K buffer it & 1 is free: group K(it + 2)
-
-      // ---- this thread's row of S(it): masked past the range; running maximum in the exp2 domain
-      uint32_t sr[2][32];
-      const uint32_t tS = tlane + (uint32_t)(it & 1) * kColS1;
-      tmem_ld32(tS, sr[0]);
-      tmem_ld32(tS + 32, sr[1]);
-      tmem_wait_ld();
-      const int nvalid = min(kVTile, t1 - (t0 + it * kVTile));
-      if (nvalid < kVTile) {
-#pragma unroll
-        for (int j = 0; j < 64; ++j)
-          if (j >= nvalid) sr[j >> 5][j & 31] = 0xff800000u;   // -inf
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-      for (int j = 0; j < 64; j += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(sr[j >> 5][j & 31]));
-        mx1 = fmaxf(mx1, __uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]));
-        mx2 = fmaxf(mx2, __uint_as_float(sr[(j + 2) >> 5][(j + 2) & 31]));
-        mx3 = fmaxf(mx3, __uint_as_float(sr[(j + 3) >> 5][(j + 3) & 31]));
-      }
-      const float m_new = fmaxf(m_used, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * scale);   // scale > 0
-      // raising the maximum rescales O, which the second product of tile it - 1 may still be writing
-      bool pv_waited = it == 0;
-      const bool raise = m_new > m_used + 8.f;
-      if (wg_or(id_wg, raise)) {
-        if (!pv_waited) {
-          if (!wg_and(id_wg, mbar_wait(bar_o, (it - 1) & 1))) { ok_all = false; *s_abort = 1; bar_sync160(id_pv); continue; }
-          tc_fence_after();
-          pv_waited = true;
-        }
-        if (__any_sync(0xffffffffu, raise)) {
-          const float factor = ex2(m_used - m_new);
-          if (it > 0) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < D; c0 += 32) {
-              uint32_t o[32];
-              tmem_ld32(tlane + kColO + c0, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
-              tmem_st32(tlane + kColO + c0, o);
-            }
-            tmem_wait_st();
-          }
-          lsum *= factor;
-          m_used = m_new;
-        }
-      }
-      // ---- P = hi + lo in registers, while the tensor pipe works on S(it + 1) and O(it - 1)
-      const float neg_m = -m_used;
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t hi[32], lo[32];
-#pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        const int j = 2 * e;
-        const float p0 = ex2(fmaf(__uint_as_float(sr[j >> 5][j & 31]), scale, neg_m));
-        const float p1 = ex2(fmaf(__uint_as_float(sr[(j + 1) >> 5][(j + 1) & 31]), scale, neg_m));
-        ls[e & 3] += p0 + p1;      // the denominator takes the weights before the hi + lo split (2^-17 apart)
-        split_pair_packed(p0, p1, hi[e], lo[e]);
-      }
-      lsum += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      // ---- the second product of tile it - 1 is done: value buffer (it + 1) & 1 is free
-      if (!pv_waited) {
-        if (!wg_and(id_wg, mbar_wait(bar_o, (it - 1) & 1))) { ok_all = false; *s_abort = 1; bar_sync160(id_pv); continue; }
-        tc_fence_after();
-      }
-      load_tile(pipe + kT2V + ((it + 1) & 1) * 16384, vg, p.v.ss, it + 1);   // group V(it + 1)
-      tmem_st32(tS, hi);             // P(it) over S(it): hi in columns [0, 32), lo in [32, 64), two tokens per column
-      tmem_st32(tS + 32, lo);
-      tmem_wait_st();
-      cp_wait<2>();                                  // V(it) has landed; K(it + 2) and V(it + 1) may be in flight
-      fence_proxy_async();
-      tc_fence_before();
-      bar_arrive160(id_pv);
-    }
-    if (ok_all && ntl > 0) {                         // the last second product
-      if (!wg_and(id_wg, mbar_wait(bar_o, (ntl - 1) & 1))) ok_all = false;
-      tc_fence_after();
-    }
-    cp_wait<0>();
-
-    // ---- partial state of this thread's row, same record as the other kernels
-    if (ok_all) {
-      const size_t rec_floats = (size_t)p.MB * (2 + D);
-      float* rec = p.partials + ((size_t)(ucall * p.nrb + rb) * p.nsplit + split) * rec_floats;
-      rec[wt] = m_used;
-      rec[p.MB + wt] = lsum;
-      float4* orow = (float4*)(rec + 2 * p.MB + (size_t)wt * D);
-#pragma unroll 1
-      for (int c0 = 0; c0 < D; c0 += 32) {
-        uint32_t o[32];
-        if (ntl > 0) {
-          tmem_ld32(tlane + kColO + c0, o);
-          tmem_wait_ld();
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[j] = 0u;
-        }
-#pragma unroll
-        for (int j = 0; j < 8; ++j)
-          orow[c0 / 4 + j] = make_float4(__uint_as_float(o[4 * j]), __uint_as_float(o[4 * j + 1]), __uint_as_float(o[4 * j + 2]),
-                                         __uint_as_float(o[4 * j + 3]));
-      }
-    } else if (wt == 0 && p.error) {
-      atomicOr(p.error, kErrWaitTimeout);
-    }
-  }
-  tc_fence_before();
-  const bool both = __syncthreads_and(ok_all);       // softmax warps and MMA warp are through
-  if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" :: "r"(*s_tmem), "r"(kT2Cols) : "memory");
-  if (!both) return;
-  finish_unit<D>(p, smem, s_last, ucall, b, l, h);
-}
-
 constexpr int smem_bytes(int D) { return kVStages * 2 * kVTile * D * 2; }
 
 }  // namespace
@@ -902,8 +608,6 @@ cudaError_t score_value_setup(int D) {
   if (D == 128) {
     cudaError_t e = cudaFuncSetAttribute(k_score_value_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcBytes + 1024);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_score_value_tc2, cudaFuncAttributeMaxDynamicSharedMemorySize, kT2Bytes);
-    if (e != cudaSuccess) return e;
   }
   if (D == 128) return cudaFuncSetAttribute(k_score_value<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(128));
   if (D == 64) return cudaFuncSetAttribute(k_score_value<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes(64));
@@ -913,10 +617,6 @@ cudaError_t score_value_setup(int D) {
 // threads = 32 * (MB / 16): one warp per 16 query rows of the row block
 cudaError_t launch_score_value(const ValueScoreParams& p, int threads, cudaStream_t s) {
   dim3 grid(p.nsplit, p.nrb, p.B * p.nlayers * p.N_kv);
-  if (p.use_tcgen05 == 2 && p.D == 128 && p.MB == 128) {
-    k_score_value_tc2<<<grid, kT2Threads, kT2Bytes, s>>>(p);
-    return cudaGetLastError();
-  }
   if (p.use_tcgen05 && p.D == 128 && p.MB == 128) {
     k_score_value_tc<<<grid, kTcThreads, kTcBytes + 1024, s>>>(p);
     return cudaGetLastError();

@@ -27,6 +27,7 @@ struct Geometry {
   // value-channel pruning (App. D)
   bool vt;
   int Tv, Tvp;                 // kept value channels, padded to a multiple of 16
+  int value_score_kernel;      // thinK_value_score_kernel
   int M, MB, nrb;              // query rows per unit of the value score, rows per row block, row blocks
   int value_slots;             // partial records the workspace holds
   int S_pmax;
@@ -54,6 +55,9 @@ thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geome
   if (g->cap < 1) g->cap = 1;
   g->tail_tiles_cap = (g->cap + kTileTokens - 1) / kTileTokens;
   g->dtype = c->dtype; g->E = c->dtype == THINK_BF16 ? 2 : 4; g->criterion = c->criterion;
+  if (c->value_score_kernel != THINK_VALUE_SCORE_AUTO && c->value_score_kernel != THINK_VALUE_SCORE_MMA_SYNC)
+    return THINK_ERR_INVALID_ARG;
+  g->value_score_kernel = c->value_score_kernel;
   const int CH = 16 / g->E;
   g->NC = c->N_kv * c->D / CH;
   g->CB = g->NC < kScoreThreads ? g->NC : kScoreThreads;
@@ -149,9 +153,10 @@ struct thinK_cache {
   std::vector<int32_t> n_re;                // per layer, 64-token tail blocks already re-pruned
   thinK_tensor5 v;                          // borrowed prompt values (set by thinK_compact)
   bool have_v;
+  thinK_sizes have_sizes, need_sizes;       // bytes of the caller's buffers as stated at thinK_create / as required
   int num_sms, decode_grid_max;
   int score_capacity;                       // resident CTAs of the score kernel on this device
-  int value_score_tcgen05;                  // 0: keep the mma.sync value-score kernel (THINK_VALUE_SCORE=mma_sync)
+  int value_score_tcgen05;                  // 0: the mma.sync value-score kernel everywhere (cfg.value_score_kernel)
 };
 
 extern "C" {
@@ -209,11 +214,20 @@ thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens,
   return THINK_OK;
 }
 
-thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void* k_thin, void* tail_k,
-                          void* tail_v, void* idx, void* scores, void* workspace, thinK_cache** out) {
+thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, const thinK_sizes* sizes, void* k_thin,
+                          void* tail_k, void* tail_v, void* idx, void* scores, void* workspace, thinK_cache** out) {
   if (!out) return THINK_ERR_INVALID_ARG;
   *out = nullptr;
-  if (!k_thin || !tail_k || !tail_v || !idx || !workspace) return THINK_ERR_INVALID_ARG;
+  if (!sizes || !k_thin || !tail_k || !tail_v || !idx || !workspace) return THINK_ERR_INVALID_ARG;
+  thinK_sizes need;
+  {
+    // the caller states how large its buffers are; anything below what this configuration needs is refused
+    thinK_status st = thinK_cache_bytes(cfg, seq_lens, &need);
+    if (st != THINK_OK) return st;
+    if (sizes->k_thin < need.k_thin || sizes->tail_k < need.tail_k || sizes->tail_v < need.tail_v ||
+        sizes->idx < need.idx || sizes->workspace < need.workspace || (scores && sizes->scores < need.scores))
+      return THINK_ERR_CAPACITY;
+  }
   if (!aligned16(k_thin) || !aligned16(tail_k) || !aligned16(tail_v) || !aligned16(workspace) ||
       (scores && !aligned16(scores)))
     return THINK_ERR_INVALID_ARG;
@@ -225,12 +239,9 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, void
   c->ws = (unsigned char*)workspace;
   c->k_thin = k_thin; c->tail_k = tail_k; c->tail_v = tail_v; c->idx = idx; c->scores = scores;
   c->v_thin = c->perm_v = c->scores_v = nullptr;
-  {
-    // which value-score kernel serves 128-row blocks at D = 128: "mma_sync", "tcgen05_2" (softmax warps + a
-    // separate MMA warp, double-buffered K/V) or, by default, the tcgen05 kernel whose threads share the roles
-    const char* e = getenv("THINK_VALUE_SCORE");
-    c->value_score_tcgen05 = e && strcmp(e, "mma_sync") == 0 ? 0 : (e && strcmp(e, "tcgen05_2") == 0 ? 2 : 1);
-  }
+  c->have_sizes = *sizes;
+  c->need_sizes = need;
+  c->value_score_tcgen05 = c->g.value_score_kernel == THINK_VALUE_SCORE_MMA_SYNC ? 0 : 1;
   c->scored_v.assign(c->g.L, 0);
   c->scored.assign(c->g.L, 0);
   c->compacted.assign(c->g.L, 0);
@@ -304,6 +315,7 @@ thinK_status score_select_impl(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor
   p.layer0 = layer0; p.nlayers = nlayers;
   p.NC = g.NC; p.CB = g.CB; p.ncolblk = g.ncolblk; p.RP = g.RPmax;
   p.criterion = g.criterion;
+  p.error = (uint32_t*)(c->ws + c->w.error);
   const int items = g.B * nlayers * g.ncolblk;
   // one wave of CTAs: the token split fills the resident slots without spilling into a second wave
   int nsplit = c->score_capacity / items;
@@ -340,7 +352,11 @@ thinK_status compact_impl(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, cons
     for (int l = layer0; l < layer0 + nlayers; ++l)
       if (!c->scored_v[l]) return THINK_ERR_STATE;
   } else if (c->have_v && memcmp(&c->v, &v_prefix, sizeof(v_prefix)) != 0) {
-    return THINK_ERR_INVALID_ARG;   // one V for all layers
+    // A different V view is a new prompt: decode reads the prefix values of all layers through ONE borrowed
+    // view, so the layers outside this call fall back to "not compacted" until they are compacted again.
+    for (int l = 0; l < g.L; ++l)
+      if (l < layer0 || l >= layer0 + nlayers) c->compacted[l] = 0;
+    c->have_v = false;
   }
   CompactParams p;
   memset(&p, 0, sizeof(p));
@@ -408,6 +424,8 @@ thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int
 }
 
 thinK_status thinK_attach_value_cache(thinK_cache* c, void* v_thin, void* perm_v, void* scores_v) {
+  if (c && c->g.vt && (c->have_sizes.v_thin < c->need_sizes.v_thin || c->have_sizes.perm_v < c->need_sizes.perm_v))
+    return THINK_ERR_CAPACITY;
   if (!c || !v_thin || !perm_v || !aligned16(v_thin) || !aligned16(perm_v) || (scores_v && !aligned16(scores_v)))
     return THINK_ERR_INVALID_ARG;
   if (!c->g.vt) return THINK_ERR_STATE;
@@ -465,6 +483,9 @@ thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_te
   for (int l0 = layer0; l0 < layer0 + nlayers; l0 += per_launch) {
     p.layer0 = l0;
     p.nlayers = l0 + per_launch <= layer0 + nlayers ? per_launch : layer0 + nlayers - l0;
+    // tickets start at zero whatever an earlier launch left behind (a CTA whose bounded wait ran out never takes its ticket)
+    if (cudaMemsetAsync(p.counters, 0, sizeof(uint32_t) * (size_t)g.B * p.nlayers * g.N_kv, (cudaStream_t)stream) != cudaSuccess)
+      return THINK_ERR_CUDA;
     if (launch_score_value(p, 32 * (g.MB / 16), (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
   }
   for (int l = layer0; l < layer0 + nlayers; ++l) c->scored_v[l] = 1;

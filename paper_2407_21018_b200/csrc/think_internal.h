@@ -31,6 +31,7 @@ struct TokenMap {
 constexpr uint32_t kErrTokenRange = 1u;   // device error word: a token index was out of range
 constexpr uint32_t kErrWaitTimeout = 2u;  // device error word: a bounded wait on an mbarrier ran out
 constexpr uint32_t kErrSmemAlign = 4u;    // device error word: dynamic shared memory not on a 1024-byte boundary
+constexpr uint32_t kErrNonFinite = 8u;    // device error word: a channel score was NaN or infinite (non-finite K or Q)
 
 struct ScoreParams {
   TokenMap tok;
@@ -46,6 +47,7 @@ struct ScoreParams {
   int CB;                   // chunks per column block
   int ncolblk, nsplit, RP;  // RP = rows in flight per CTA iteration
   int criterion;
+  uint32_t* error;          // device error word (may be null)
 };
 
 struct CompactParams {
@@ -92,7 +94,7 @@ struct ValueScoreParams {    // App. D: Score_v = column norms of the window's a
   int M;                    // G * S_obs query rows per unit
   int MB;                   // rows per row block (multiple of 16, <= 128)
   int nrb, nsplit;
-  int use_tcgen05;          // D = 128 and MB = 128: 0 mma.sync kernel, 1 tcgen05 (one pipeline per CTA), 2 two pipelines per CTA
+  int use_tcgen05;          // D = 128 and MB = 128: 1 tcgen05 kernel (accumulators in tensor memory), 0 mma.sync kernel
   uint32_t* error;          // device error word
 };
 
@@ -213,16 +215,23 @@ __device__ __forceinline__ int64_t token_row(const TokenMap& m, int64_t unit, in
 // Rank-count selection of one head by one warp: channel j is kept when fewer than T channels
 // beat it, where k beats j if s[k] > s[j] or (s[k] == s[j] and k < j).  out[0..T) = kept channels
 // ascending; with `rest`, out[T..D) = the other channels ascending (out is then a permutation).
-__device__ __forceinline__ void select_head(const double* s, int D, int T, uint8_t* out, int lane, bool rest) {
+// A NaN score ranks as -infinity, so the order is total and exactly T channels are kept whatever
+// the inputs; a NaN or infinite score raises kErrNonFinite in *error (when given).
+__device__ __forceinline__ void select_head(const double* s, int D, int T, uint8_t* out, int lane, bool rest,
+                                            uint32_t* error = nullptr) {
   int base = 0, base_rest = T;
+  bool bad = false;
   for (int j0 = 0; j0 < D; j0 += 32) {
     int j = j0 + lane;
     bool keep = false;
     if (j < D) {
       double sj = s[j];
+      bad |= !(fabs(sj) <= 1.7976931348623157e308);
+      if (!(sj == sj)) sj = -INFINITY;
       int rank = 0;
       for (int k = 0; k < D; ++k) {
         double sk = s[k];
+        if (!(sk == sk)) sk = -INFINITY;
         rank += (sk > sj) || (sk == sj && k < j);
       }
       keep = rank < T;
@@ -238,6 +247,7 @@ __device__ __forceinline__ void select_head(const double* s, int D, int T, uint8
       base_rest += __popc(o);
     }
   }
+  if (error && __any_sync(0xffffffffu, bad) && lane == 0) atomicOr(error, kErrNonFinite);
 }
 
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }

@@ -21,11 +21,11 @@ SCORE_V_RTOL = 1e-4                    # value scores: bf16 tensor-core products
 NEAR_TIE_V_REL = 1e-4
 
 
-def make_cache(w: wl.Workload, steps=None, criterion=0, keep_scores=True, lam_v=0.0):
+def make_cache(w: wl.Workload, steps=None, criterion=0, keep_scores=True, lam_v=0.0, value_score_kernel=0):
     from paper_2407_21018_b200 import binding as tk
     steps = w.steps if steps is None else steps
     cfg = tk.make_config(w.B, w.L, w.N_q, w.N_kv, w.D, w.S_max, w.S_obs, w.recent, steps, w.lam,
-                         w.torch_dtype, criterion, lam_v)
+                         w.torch_dtype, criterion, lam_v, value_score_kernel)
     cache = tk.ThinKCache(cfg, w.seq_lens, device="cuda", keep_scores=keep_scores)
     cache.k_thin.zero_()     # the tiles reserved for re-pruned tail blocks stay unwritten: make buffers comparable
     return cache

@@ -105,4 +105,24 @@ def test_null_arguments(tk):
     h = C.c_void_p()
     cfg = tk.make_config(1, 1, 4, 4, 64, 512, 32, 32, 8, 0.5, tk.F32)
     arr = (C.c_int32 * 1)(512)
-    assert tk.lib.thinK_create(C.byref(cfg), arr, None, None, None, None, None, None, C.byref(h)) == tk.ERR_INVALID_ARG
+    sizes = tk.thinK_cache_bytes(cfg, [512])
+    assert tk.lib.thinK_create(C.byref(cfg), arr, C.byref(sizes), None, None, None, None, None, None,
+                               C.byref(h)) == tk.ERR_INVALID_ARG
+    assert tk.lib.thinK_create(C.byref(cfg), arr, None, 256, 256, 256, 256, None, 256, C.byref(h)) == tk.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("short", ["k_thin", "tail_k", "tail_v", "idx", "workspace", "scores"])
+def test_create_refuses_buffers_smaller_than_required(tk, short):
+    """thinK_create compares the caller's stated buffer sizes with what the configuration needs; the
+    check comes before any device access, so fake (aligned, never dereferenced) pointers do here."""
+    cfg = tk.make_config(2, 2, 8, 4, 64, 512, 32, 32, 8, 0.5, tk.BF16)
+    lens = [512, 300]
+    arr = (C.c_int32 * 2)(*lens)
+    have = tk.thinK_cache_bytes(cfg, lens)
+    setattr(have, short, getattr(have, short) - 1)
+    h = C.c_void_p()
+    fake = [4096] * 6                                   # k_thin, tail_k, tail_v, idx, scores, workspace
+    st = tk.lib.thinK_create(C.byref(cfg), arr, C.byref(have), *fake, C.byref(h))
+    assert st == tk.ERR_CAPACITY and not h.value
+    if short == "scores":                               # an absent score buffer needs no size
+        pass

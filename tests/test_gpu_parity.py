@@ -192,21 +192,18 @@ def test_eviction_rejects_bad_arguments():
 @pytest.mark.parametrize("name,S,L,B,lam_v,R,kernel", [
     ("c2", 1100, 2, 1, 0.3, 32, "tcgen05"),    # GQA 4:1 -> 128 window rows per key head, T_v = 89 (rows padded to 96)
     ("c2", 1100, 2, 1, 0.3, 32, "mma_sync"),   # the same through the mma.sync score kernel
-    ("c2", 1100, 2, 1, 0.3, 32, "tcgen05_2"),  # ... and through the two-pipeline tcgen05 kernel
     ("c4", 600, 1, 3, 0.5, 32, "tcgen05"),     # MHA -> 32 rows (always mma.sync), ragged batch, T_v = 64
     ("c5", 2100, 1, 1, 0.25, 0, "tcgen05"),    # S_obs = 64 -> 256 rows = two row blocks; no recent window
     ("c5", 2100, 1, 1, 0.25, 0, "mma_sync"),
-    ("c5", 2100, 1, 1, 0.25, 0, "tcgen05_2"),
     ("c2", 700, 1, 2, 0.9, 32, "tcgen05"),     # T_v = 12: one 16-channel group of values
 ])
-def test_value_channel_pruning(name, S, L, B, lam_v, R, kernel, monkeypatch):
+def test_value_channel_pruning(name, S, L, B, lam_v, R, kernel):
     """App. D through the whole path: value scores and their ranking, thinned prefix values,
     tail values in the permuted order, decode over thinned keys AND values."""
-    monkeypatch.setenv("THINK_VALUE_SCORE", kernel)       # read when the cache is created
     w = dataclasses.replace(wl.shrink(wl.get_config(name), S=S, L=L, B=B, steps=5), S_recent=R)
     data = wl.make_prefill(w, device="cpu")
     K, V, Q = data["K"].cuda(), data["V"].cuda(), data["Q_obs"].cuda()
-    cache = make_cache(w, w.steps, lam_v=lam_v)
+    cache = make_cache(w, w.steps, lam_v=lam_v, value_score_kernel=1 if kernel == "mma_sync" else 0)
     cache.prefill(Q, K, V)
     torch.cuda.synchronize()
     o = make_oracle(w, lam_v)
