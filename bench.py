@@ -172,9 +172,11 @@ def run_ours(args):
         elif Tv:
             cache.score_select_kv(Q, K, V)
             cache.compact(K, V)
-        else:
+        elif args.two_pass_prefill:
             cache.score_select(Q, K)
             cache.compact(K, V)
+        else:
+            cache.prefill(Q, K, V)
         if ev is not None:
             ev["p1"].record(stream)
         for t in range(nsteps):
@@ -453,6 +455,8 @@ def main():
                     help="decode steps through thinK_append_decode (append + attention in one call, the attention "
                          "launched as a programmatic dependent); decode.us_per_step is then the whole step")
     ap.add_argument("--lam", type=float, default=None, help="override the config's pruning ratio (c5 sweep)")
+    ap.add_argument("--two-pass-prefill", action="store_true",
+                    help="prefill through thinK_score_select + thinK_compact (two passes over K) instead of thinK_prefill")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=15.0)

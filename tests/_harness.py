@@ -40,9 +40,11 @@ def bf16_ulp(x: np.ndarray) -> np.ndarray:
     return 2.0 ** (np.floor(np.log2(ax)) - 7)
 
 
-def assert_attn_close(gpu: np.ndarray, want: np.ndarray, dtype: str, where=""):
-    """fp32 I/O: max-abs <= 1e-5.  bf16 I/O: max-abs <= 1e-2 wherever the bf16 grid allows it
-    (|x| < 4: half an ulp is below 1e-2); larger outputs must be within one bf16 ulp."""
+def assert_attn_close(gpu: np.ndarray, want: np.ndarray, dtype: str, where="", stats=None):
+    """fp32 I/O: max-abs <= 1e-5.  bf16 I/O: max-abs <= 1e-2 for |x| < 4.  A bf16 output of magnitude >= 4
+    cannot meet 1e-2 by construction (half an ulp there is 0.0156 or more), so those elements must lie
+    within half a bf16 ulp + 1e-3 of the oracle; `stats["large"]` counts them (the c1-c5 workloads have
+    none: their values are N(0, 1) and the outputs convex combinations of them)."""
     assert np.isfinite(gpu).all(), f"non-finite output {where}"
     err = np.abs(gpu - want)
     if dtype == "f32":
@@ -52,8 +54,36 @@ def assert_attn_close(gpu: np.ndarray, want: np.ndarray, dtype: str, where=""):
     if small.any():
         assert err[small].max() <= ATOL["bf16"], f"{where}: max-abs {err[small].max():.3e}"
     if (~small).any():
-        assert (err[~small] <= bf16_ulp(want[~small])).all(), f"{where}: large outputs off by more than an ulp"
+        bar = 0.5 * bf16_ulp(want[~small]) + 1e-3
+        assert (err[~small] <= bar).all(), f"{where}: large outputs off by more than half an ulp + 1e-3"
+    if stats is not None:
+        stats["large"] = stats.get("large", 0) + int((~small).sum())
+        stats["max_abs"] = max(stats.get("max_abs", 0.0), float(err.max()))
     return float(err.max())
+
+
+def check_head_selection(got: np.ndarray, score: np.ndarray, T: int, band: float, where="") -> int:
+    """One head's kept channels against Top_T of the oracle's scores: 0 when identical; 1 when they differ
+    but the oracle's own scores at the cut are a near-tie (relative gap < band) AND the disagreement is
+    confined to channels whose scores lie inside that band.  Anything else fails."""
+    got = np.asarray(got, dtype=np.int64)
+    assert (np.diff(got) > 0).all(), f"{where} idx not ascending"
+    want = orc.select_top_T(score, T)
+    if (got == want).all():
+        return 0
+    assert orc.near_tie(score, T, band), f"{where} idx mismatch without a near-tie"
+    cut = np.sort(score)[::-1][T - 1]
+    diff = set(got.tolist()) ^ set(want.tolist())
+    assert all(abs(score[j] - cut) <= 2 * band * cut for j in diff), f"{where} idx mismatch outside the near-tie band"
+    return 1
+
+
+# statistics the parity tests leave for the end-of-run summary (tests/conftest.py prints them)
+PARITY_STATS = []
+
+
+def record_parity(name: str, **kw):
+    PARITY_STATS.append(dict(case=name, **kw))
 
 
 def compare_selection(idx_gpu: np.ndarray, score_gpu, o: orc.ThinKOracle, where="", values=False):
@@ -69,21 +99,15 @@ def compare_selection(idx_gpu: np.ndarray, score_gpu, o: orc.ThinKOracle, where=
     for b in range(B):
         for l in range(L):
             for h in range(N):
-                got, want = idx_gpu[b, l, h].astype(np.int64), o_idx[b, l, h]
-                assert (np.diff(got) > 0).all(), f"{where} idx not ascending at {(b, l, h)}"
+                got = idx_gpu[b, l, h].astype(np.int64)
                 if score_gpu is not None:
                     np.testing.assert_allclose(score_gpu[b, l, h], o_score[b, l, h], rtol=s_rtol,
                                                err_msg=f"{where} scores at {(b, l, h)}")
-                if (got == want).all():
-                    continue
-                s = o_score[b, l, h]
-                assert orc.near_tie(s, T, band), f"{where} idx mismatch at {(b, l, h)} without a near-tie"
-                cut = np.sort(s)[::-1][T - 1]
-                diff = set(got.tolist()) ^ set(want.tolist())
-                assert all(abs(s[j] - cut) <= 2 * band * cut for j in diff), \
-                    f"{where} idx mismatch outside the near-tie band at {(b, l, h)}"
-                o_idx[b, l, h] = got
-                near += 1
+                if check_head_selection(got, o_score[b, l, h], T, band, f"{where} {(b, l, h)}"):
+                    o_idx[b, l, h] = got
+                    near += 1
+    if near:
+        record_parity(where + (" values" if values else ""), near_ties=near, heads=B * L * N)
     return near
 
 

@@ -24,3 +24,16 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Parity statistics gathered by the GPU tests: near-tie heads, index mismatches, max-abs errors."""
+    try:
+        from _harness import PARITY_STATS
+    except Exception:
+        return
+    if PARITY_STATS:
+        import json
+        terminalreporter.write_sep("-", "parity statistics")
+        for rec in PARITY_STATS:
+            terminalreporter.write_line("PARITY " + json.dumps(rec))
