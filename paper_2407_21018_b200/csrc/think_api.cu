@@ -15,7 +15,7 @@ namespace {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // byte offsets inside the workspace
-  size_t seq_len, cum_thin, thin_tile_base, error, v_thin_base, score_counters, decode_counters;
+  size_t seq_len, cum_thin, thin_tile_base, error, v_thin_base, row_cum, score_counters, decode_counters;
   size_t score_partials, decode_records, total;
   size_t value_counters, value_partials;   // value-channel scoring (only with lambda_v > 0)
   size_t header_bytes;     // everything before score_partials (initialised by thinK_create)
@@ -35,7 +35,7 @@ struct Geometry {
   int64_t total_thin_tiles;    // over all (b, l, h)
   int max_thin_tiles;          // per (l, h) over b
   std::vector<int32_t> seq_len, cum_thin;
-  std::vector<int64_t> thin_tile_base;
+  std::vector<int64_t> thin_tile_base, row_cum;
 };
 
 thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geometry* g) {
@@ -66,12 +66,14 @@ thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geome
   g->seq_len.assign(seq_lens, seq_lens + c->B);
   g->cum_thin.assign(c->B + 1, 0);
   g->thin_tile_base.assign(c->B + 1, 0);
+  g->row_cum.assign(c->B + 1, 0);
   g->max_thin_tiles = 0;
   for (int b = 0; b < c->B; ++b) {
     const int S = seq_lens[b];
     if (S < c->S_obs || S < c->S_recent || S > c->S_max || S < 1) return THINK_ERR_INVALID_ARG;
     const int nt = (S - c->S_recent + kTileTokens - 1) / kTileTokens;
     g->cum_thin[b + 1] = g->cum_thin[b] + nt;
+    g->row_cum[b + 1] = g->row_cum[b] + S;
     g->thin_tile_base[b + 1] = g->thin_tile_base[b] + (int64_t)c->L * c->N_kv * (nt + g->tail_tiles_cap);
     if (nt > g->max_thin_tiles) g->max_thin_tiles = nt;
   }
@@ -111,6 +113,7 @@ void make_layout(const Geometry& g, Layout* w) {
   w->thin_tile_base = o;   o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
   w->error = o;            o = align_up(o + 256, 256);
   w->v_thin_base = o;      o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
+  w->row_cum = o;          o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
   w->score_counters = o;   o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.ncolblk, 256);
   w->decode_counters = o;  o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.N_kv, 256);
   w->value_counters = o;
@@ -156,6 +159,7 @@ struct thinK_cache {
   thinK_sizes have_sizes, need_sizes;       // bytes of the caller's buffers as stated at thinK_create / as required
   int num_sms, decode_grid_max;
   int score_capacity;                       // resident CTAs of the score kernel on this device
+  int score_flat_capacity;                  // ... of the flat-partition score kernel
   int value_score_tcgen05;                  // 0: the mma.sync value-score kernel everywhere (cfg.value_score_kernel)
 };
 
@@ -264,6 +268,9 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, cons
   if (c->decode_grid_max * wpc > kMaxDecodeCtas) c->decode_grid_max = kMaxDecodeCtas / wpc;
   c->score_capacity = c->num_sms * score_ctas_per_sm(c->g.dtype, c->g.criterion);
   if (c->score_capacity < 1) { delete c; return THINK_ERR_CUDA; }
+  c->score_flat_capacity = c->num_sms * score_flat_ctas_per_sm(c->g.dtype, c->g.criterion);
+  if (c->score_flat_capacity < 1) { delete c; return THINK_ERR_CUDA; }
+  if (c->score_flat_capacity > kScoreTargetCtas / 2) c->score_flat_capacity = kScoreTargetCtas / 2;   // two partial slots each
   // device tables
   const Geometry& g = c->g;
   bool ok = cudaMemset(c->ws, 0, c->w.header_bytes) == cudaSuccess;
@@ -271,6 +278,7 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, cons
   ok = ok && cudaMemcpy(c->ws + c->w.cum_thin, g.cum_thin.data(), sizeof(int32_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->ws + c->w.thin_tile_base, g.thin_tile_base.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->ws + c->w.v_thin_base, g.v_thin_base.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->ws + c->w.row_cum, g.row_cum.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   if (!ok) { delete c; return THINK_ERR_CUDA; }
   *out = c;
   return THINK_OK;
@@ -316,8 +324,19 @@ thinK_status score_select_impl(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor
   p.NC = g.NC; p.CB = g.CB; p.ncolblk = g.ncolblk; p.RP = g.RPmax;
   p.criterion = g.criterion;
   p.error = (uint32_t*)(c->ws + c->w.error);
+  if (!tok.rows) {
+    // prompt order: all (b, layer, column block) items end to end, cut into equal pieces over one full wave
+    p.row_cum = (const int64_t*)(c->ws + c->w.row_cum);
+    p.flat_rows = (long long)nlayers * g.ncolblk * g.row_cum[g.B];
+    long long grid = p.flat_rows / (16 * p.RP);            // at least 16 rows per row lane and piece
+    if (grid > c->score_flat_capacity) grid = c->score_flat_capacity;
+    if (grid < 1) grid = 1;
+    if (launch_score_flat(p, g.dtype, (int)grid, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
+    for (int l = layer0; l < layer0 + nlayers; ++l) c->scored[l] = 1;
+    return THINK_OK;
+  }
   const int items = g.B * nlayers * g.ncolblk;
-  // one wave of CTAs: the token split fills the resident slots without spilling into a second wave
+  // kept-token lists: one wave of CTAs, the token split fills the resident slots without spilling into a second wave
   int nsplit = c->score_capacity / items;
   if (nsplit > (kScoreTargetCtas + items - 1) / items) nsplit = (kScoreTargetCtas + items - 1) / items;
   // keep at least 64 token rows per row lane of a split

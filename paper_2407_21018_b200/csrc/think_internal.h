@@ -48,6 +48,9 @@ struct ScoreParams {
   int ncolblk, nsplit, RP;  // RP = rows in flight per CTA iteration
   int criterion;
   uint32_t* error;          // device error word (may be null)
+  // k_colnorm_flat only: all items laid end to end, one unit per token row
+  const int64_t* row_cum;   // [B + 1] prompt rows of the batch entries before b
+  long long flat_rows;      // nlayers * ncolblk * row_cum[B]
 };
 
 struct CompactParams {
@@ -157,6 +160,8 @@ struct DecodeParams {
 // launchers (one per translation unit); return the launch status
 cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s);
 int score_ctas_per_sm(int dtype, int criterion);
+cudaError_t launch_score_flat(const ScoreParams& p, int dtype, int grid, cudaStream_t s);
+int score_flat_ctas_per_sm(int dtype, int criterion);
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s);
 cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s, bool overlap_previous = false);
 cudaError_t launch_reprune(const RepruneParams& p, cudaStream_t s);

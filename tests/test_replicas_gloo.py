@@ -38,3 +38,16 @@ def test_single_replica_needs_no_group():
     sys.path.insert(0, ROOT)
     from paper_2407_21018_b200 import replicas
     assert replicas.job_time_and_work(3.0, 7.0) == (3.0, 7.0)
+
+
+def test_launch_starts_the_asked_number_of_ranks(tmp_path):
+    """The path `bench.py --gpus N` takes when it is started as ONE process: it re-launches itself as N
+    ranks through replicas.launch.  Here the ranks are CPU processes on gloo."""
+    sys.path.insert(0, ROOT)
+    from paper_2407_21018_b200 import replicas
+    out = tmp_path / "ranks.txt"
+    rc = replicas.launch(2, os.path.join(ROOT, "tests", "_replica_probe.py"), [str(out)],
+                         port=31000 + os.getpid() % 2000)
+    assert rc == 0
+    world, ms, units = out.read_text().split()
+    assert int(world) == 2 and float(ms) == 20.0 and float(units) == 2.0
