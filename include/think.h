@@ -298,7 +298,12 @@ thinK_status thinK_score_select_static(const thinK_config* cfg, const int32_t* s
  * not an error (nothing happens).  The values of the moved tokens stay where they are (tail_v).
  * Attention afterwards treats those tokens like prefix tokens: gathered query x thinned keys.
  * bf16 caches only (THINK_ERR_UNSUPPORTED otherwise).  All layers of a decode call must have been
- * re-pruned alike. */
+ * re-pruned alike.
+ * What it saves is HBM traffic per decode step (the moved keys are read at T channels instead of D) and,
+ * in the paper's accounting, cache size; it gives no ALLOCATED memory back: tail_k and tail_v stay sized
+ * for S_recent + max_new_tokens full-width rows, positions keep counting against that capacity, and
+ * k_thin carries ceil(cap/64) spare tiles per head for the moved blocks whether or not they are used.
+ * thinK_sizes.model_think_bytes does not account for re-pruning. */
 thinK_status thinK_reprune_tail(thinK_cache* c, int32_t keep_recent, int32_t layer0, int32_t nlayers, void* stream);
 
 /* Tokens of the tail buffers of `layer` whose keys have been re-pruned (a multiple of 64), or -1. */

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libthink.so")
-SOURCES = ["think_api.cu", "k_score.cu", "k_score_flat.cu", "k_score_value.cu", "k_compact.cu", "k_decode.cu", "k_decode_mma.cu"]
+SOURCES = ["think_api.cu", "k_score.cu", "k_score_value.cu", "k_compact.cu", "k_decode.cu", "k_decode_mma.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]

@@ -83,13 +83,25 @@ __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
   const int pitch = D * 2 + 16;
   unsigned char* s_in = smem;                                   // [64][pitch]
   uint8_t* s_idx = smem + kTileTokens * pitch;                  // [Tp], padding channels -> 255
-  const int zb = gridDim.z - 1 - blockIdx.z;                    // last layers first: their keys are the
-  const int h = blockIdx.y;                                     // most recently scored, likely still in L2
-  const int b = zb / p.nlayers, l = p.layer0 + zb % p.nlayers;
+  // Which CTAs run side by side.  heads_first: the same 64 tokens of neighbouring heads and layers -- in the
+  // paper's B x S x L x N x D layout those rows are one contiguous stretch (L*N*D elements per token), which
+  // pays when that stretch is short (grouped-query shapes).  Otherwise: consecutive tiles of one head, whose
+  // thinned tiles are contiguous in k_thin, which pays when a token's keys span many heads (MHA).
+  int tile_i, h, l;
+  if (p.heads_first) {
+    h = blockIdx.x % p.N_kv;
+    l = p.layer0 + blockIdx.x / p.N_kv;
+    tile_i = blockIdx.y;
+  } else {
+    tile_i = blockIdx.x % p.max_tiles;
+    h = blockIdx.x / p.max_tiles;
+    l = p.layer0 + blockIdx.y;
+  }
+  const int b = blockIdx.z;
   const int S_p = p.seq_len[b] - p.R;
   const int ntiles = (S_p + kTileTokens - 1) / kTileTokens;
-  if ((int)blockIdx.x >= ntiles) return;
-  const int tile = ntiles - 1 - blockIdx.x;
+  if (tile_i >= ntiles) return;
+  const int tile = tile_i;
   const int tok0 = tile * kTileTokens;
   const int nvalid = min(kTileTokens, S_p - tok0);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -329,8 +341,10 @@ cudaError_t launch_gather_rows(const GatherRowsParams& p, int dtype, cudaStream_
   return cudaGetLastError();
 }
 
-cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s) {
+cudaError_t launch_compact(const CompactParams& p_in, int dtype, int max_tiles, cudaStream_t s) {
   if (max_tiles <= 0) return cudaSuccess;
+  CompactParams p = p_in;
+  p.max_tiles = max_tiles;
   dim3 grid(max_tiles, p.N_kv, p.B * p.nlayers);
   const int E = dtype == THINK_BF16 ? 2 : 4;
   size_t smem = (size_t)kTileTokens * (p.D * E + 16) + (size_t)p.Tp * kTileTokens * E + ((p.T + 15) & ~15);
@@ -338,7 +352,9 @@ cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cud
   if (dtype == THINK_BF16) {
     smem = (size_t)kTileTokens * (p.D * 2 + 16) + ((p.Tp + 15) & ~15);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
+    if (p.B > 65535 || p.nlayers > 65535) return cudaErrorInvalidValue;
+    p.heads_first = p.N_kv * p.nlayers <= 256 && max_tiles <= 65535;
+    cfg.gridDim = p.heads_first ? dim3(p.N_kv * p.nlayers, max_tiles, p.B) : dim3(p.N_kv * max_tiles, p.nlayers, p.B);
     cfg.blockDim = dim3(128);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;

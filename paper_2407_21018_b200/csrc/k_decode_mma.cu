@@ -14,7 +14,8 @@
 //    query heads of the group are the rows of A (rows G..15 are zero), the 16 tokens of the step are
 //    the columns of q.K^T and the contraction index of p.V.  The CUDA-core formulation needs about
 //    5.5 instructions per key/value element for G = 4, which by itself exceeds the issue slots
-//    available in the time HBM needs to deliver the bytes (profiles/k_decode_generic_c2_ncu.md).
+//    available in the time HBM needs to deliver the bytes (measured: 146.6 M warp instructions per launch of
+//    the CUDA-core kernel on the LLaMA-3-8B-shaped workload against 41.5 M here).
 //  * online softmax per step in the exp2 domain; partial states of units shared by several workers
 //    go to the workspace and the worker that arrives last at the unit's ticket merges them.
 #include <math.h>

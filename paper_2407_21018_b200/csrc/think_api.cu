@@ -6,16 +6,26 @@
 #include <new>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "think_internal.h"
 
 using namespace think;
+
+namespace {
+// NVTX range around an entry point (shows the ABI calls on a profiler's timeline; a no-op without a tool attached)
+struct Range {
+  explicit Range(const char* name) { nvtxRangePushA(name); }
+  ~Range() { nvtxRangePop(); }
+};
+}  // namespace
 
 namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {            // byte offsets inside the workspace
-  size_t seq_len, cum_thin, thin_tile_base, error, v_thin_base, row_cum, score_counters, decode_counters;
+  size_t seq_len, cum_thin, thin_tile_base, error, v_thin_base, score_counters, decode_counters;
   size_t score_partials, decode_records, total;
   size_t value_counters, value_partials;   // value-channel scoring (only with lambda_v > 0)
   size_t header_bytes;     // everything before score_partials (initialised by thinK_create)
@@ -35,7 +45,7 @@ struct Geometry {
   int64_t total_thin_tiles;    // over all (b, l, h)
   int max_thin_tiles;          // per (l, h) over b
   std::vector<int32_t> seq_len, cum_thin;
-  std::vector<int64_t> thin_tile_base, row_cum;
+  std::vector<int64_t> thin_tile_base;
 };
 
 thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geometry* g) {
@@ -66,14 +76,12 @@ thinK_status make_geometry(const thinK_config* c, const int32_t* seq_lens, Geome
   g->seq_len.assign(seq_lens, seq_lens + c->B);
   g->cum_thin.assign(c->B + 1, 0);
   g->thin_tile_base.assign(c->B + 1, 0);
-  g->row_cum.assign(c->B + 1, 0);
   g->max_thin_tiles = 0;
   for (int b = 0; b < c->B; ++b) {
     const int S = seq_lens[b];
     if (S < c->S_obs || S < c->S_recent || S > c->S_max || S < 1) return THINK_ERR_INVALID_ARG;
     const int nt = (S - c->S_recent + kTileTokens - 1) / kTileTokens;
     g->cum_thin[b + 1] = g->cum_thin[b] + nt;
-    g->row_cum[b + 1] = g->row_cum[b] + S;
     g->thin_tile_base[b + 1] = g->thin_tile_base[b] + (int64_t)c->L * c->N_kv * (nt + g->tail_tiles_cap);
     if (nt > g->max_thin_tiles) g->max_thin_tiles = nt;
   }
@@ -113,7 +121,6 @@ void make_layout(const Geometry& g, Layout* w) {
   w->thin_tile_base = o;   o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
   w->error = o;            o = align_up(o + 256, 256);
   w->v_thin_base = o;      o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
-  w->row_cum = o;          o = align_up(o + sizeof(int64_t) * (g.B + 1), 256);
   w->score_counters = o;   o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.ncolblk, 256);
   w->decode_counters = o;  o = align_up(o + sizeof(uint32_t) * (size_t)g.B * g.L * g.N_kv, 256);
   w->value_counters = o;
@@ -159,7 +166,6 @@ struct thinK_cache {
   thinK_sizes have_sizes, need_sizes;       // bytes of the caller's buffers as stated at thinK_create / as required
   int num_sms, decode_grid_max;
   int score_capacity;                       // resident CTAs of the score kernel on this device
-  int score_flat_capacity;                  // ... of the flat-partition score kernel
   int value_score_tcgen05;                  // 0: the mma.sync value-score kernel everywhere (cfg.value_score_kernel)
 };
 
@@ -220,6 +226,7 @@ thinK_status thinK_cache_bytes(const thinK_config* cfg, const int32_t* seq_lens,
 
 thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, const thinK_sizes* sizes, void* k_thin,
                           void* tail_k, void* tail_v, void* idx, void* scores, void* workspace, thinK_cache** out) {
+  Range nvtx_range("thinK_create");
   if (!out) return THINK_ERR_INVALID_ARG;
   *out = nullptr;
   if (!sizes || !k_thin || !tail_k || !tail_v || !idx || !workspace) return THINK_ERR_INVALID_ARG;
@@ -268,9 +275,6 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, cons
   if (c->decode_grid_max * wpc > kMaxDecodeCtas) c->decode_grid_max = kMaxDecodeCtas / wpc;
   c->score_capacity = c->num_sms * score_ctas_per_sm(c->g.dtype, c->g.criterion);
   if (c->score_capacity < 1) { delete c; return THINK_ERR_CUDA; }
-  c->score_flat_capacity = c->num_sms * score_flat_ctas_per_sm(c->g.dtype, c->g.criterion);
-  if (c->score_flat_capacity < 1) { delete c; return THINK_ERR_CUDA; }
-  if (c->score_flat_capacity > kScoreTargetCtas / 2) c->score_flat_capacity = kScoreTargetCtas / 2;   // two partial slots each
   // device tables
   const Geometry& g = c->g;
   bool ok = cudaMemset(c->ws, 0, c->w.header_bytes) == cudaSuccess;
@@ -278,7 +282,6 @@ thinK_status thinK_create(const thinK_config* cfg, const int32_t* seq_lens, cons
   ok = ok && cudaMemcpy(c->ws + c->w.cum_thin, g.cum_thin.data(), sizeof(int32_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->ws + c->w.thin_tile_base, g.thin_tile_base.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->ws + c->w.v_thin_base, g.v_thin_base.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
-  ok = ok && cudaMemcpy(c->ws + c->w.row_cum, g.row_cum.data(), sizeof(int64_t) * (g.B + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   if (!ok) { delete c; return THINK_ERR_CUDA; }
   *out = c;
   return THINK_OK;
@@ -324,19 +327,8 @@ thinK_status score_select_impl(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor
   p.NC = g.NC; p.CB = g.CB; p.ncolblk = g.ncolblk; p.RP = g.RPmax;
   p.criterion = g.criterion;
   p.error = (uint32_t*)(c->ws + c->w.error);
-  if (!tok.rows) {
-    // prompt order: all (b, layer, column block) items end to end, cut into equal pieces over one full wave
-    p.row_cum = (const int64_t*)(c->ws + c->w.row_cum);
-    p.flat_rows = (long long)nlayers * g.ncolblk * g.row_cum[g.B];
-    long long grid = p.flat_rows / (16 * p.RP);            // at least 16 rows per row lane and piece
-    if (grid > c->score_flat_capacity) grid = c->score_flat_capacity;
-    if (grid < 1) grid = 1;
-    if (launch_score_flat(p, g.dtype, (int)grid, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
-    for (int l = layer0; l < layer0 + nlayers; ++l) c->scored[l] = 1;
-    return THINK_OK;
-  }
   const int items = g.B * nlayers * g.ncolblk;
-  // kept-token lists: one wave of CTAs, the token split fills the resident slots without spilling into a second wave
+  // one wave of CTAs: the token split fills the resident slots without spilling into a second wave
   int nsplit = c->score_capacity / items;
   if (nsplit > (kScoreTargetCtas + items - 1) / items) nsplit = (kScoreTargetCtas + items - 1) / items;
   // keep at least 64 token rows per row lane of a split
@@ -434,11 +426,13 @@ extern "C" {
 
 thinK_status thinK_score_select(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, int32_t layer0,
                                 int32_t nlayers, void* stream) {
+  Range nvtx_range("thinK_score_select");
   return score_select_impl(c, q_obs, k, kNoTokenMap, layer0, nlayers, stream);
 }
 
 thinK_status thinK_compact(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0, int32_t nlayers,
                            void* stream) {
+  Range nvtx_range("thinK_compact");
   return compact_impl(c, k, v, kNoTokenMap, v, layer0, nlayers, stream);
 }
 
@@ -456,6 +450,7 @@ thinK_status thinK_attach_value_cache(thinK_cache* c, void* v_thin, void* perm_v
 
 thinK_status thinK_score_select_kv(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v,
                                    int32_t layer0, int32_t nlayers, void* stream) {
+  Range nvtx_range("thinK_score_select_kv");
   if (!c) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   const Geometry& g = c->g;
@@ -520,6 +515,7 @@ size_t thinK_v_kept_bytes(const thinK_cache* c) {
 thinK_status thinK_prefill_evicted(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v,
                                    const int32_t* tok, int64_t tok_stride, int32_t src_tokens, void* v_kept,
                                    int32_t layer0, int32_t nlayers, void* stream) {
+  Range nvtx_range("thinK_prefill_evicted");
   if (!c || !v_kept || !aligned16(v_kept)) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   const Geometry& g = c->g;
@@ -548,6 +544,7 @@ thinK_status thinK_prefill_evicted(thinK_cache* c, thinK_tensor5 q_obs, thinK_te
 
 thinK_status thinK_prefill(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k, thinK_tensor5 v, int32_t layer0,
                            int32_t nlayers, void* stream) {
+  Range nvtx_range("thinK_prefill");
   if (!c) return THINK_ERR_INVALID_ARG;
   thinK_status st = c->g.vt ? thinK_score_select_kv(c, q_obs, k, v, layer0, nlayers, stream)
                             : thinK_score_select(c, q_obs, k, layer0, nlayers, stream);
@@ -557,6 +554,7 @@ thinK_status thinK_prefill(thinK_cache* c, thinK_tensor5 q_obs, thinK_tensor5 k,
 
 thinK_status thinK_append(thinK_cache* c, const void* k_new, const void* v_new, int32_t layer0, int32_t nlayers,
                           void* stream) {
+  Range nvtx_range("thinK_append");
   if (!c || !k_new || !v_new) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   if (!aligned16(k_new) || !aligned16(v_new)) return THINK_ERR_INVALID_ARG;
@@ -629,11 +627,13 @@ static thinK_status decode_impl(thinK_cache* c, const void* q, void* out, int32_
 
 thinK_status thinK_decode_attn(thinK_cache* c, const void* q, void* out, int32_t layer0, int32_t nlayers,
                                void* stream) {
+  Range nvtx_range("thinK_decode_attn");
   return decode_impl(c, q, out, layer0, nlayers, stream, false);
 }
 
 thinK_status thinK_append_decode(thinK_cache* c, const void* k_new, const void* v_new, const void* q, void* out,
                                  int32_t layer0, int32_t nlayers, void* stream) {
+  Range nvtx_range("thinK_append_decode");
   if (!c || !q || !out || !aligned16(q) || !aligned16(out)) return THINK_ERR_INVALID_ARG;   // nothing launched
   thinK_status st = thinK_append(c, k_new, v_new, layer0, nlayers, stream);
   if (st != THINK_OK) return st;
@@ -641,6 +641,7 @@ thinK_status thinK_append_decode(thinK_cache* c, const void* k_new, const void* 
 }
 
 thinK_status thinK_reprune_tail(thinK_cache* c, int32_t keep_recent, int32_t layer0, int32_t nlayers, void* stream) {
+  Range nvtx_range("thinK_reprune_tail");
   if (!c || keep_recent < 0) return THINK_ERR_INVALID_ARG;
   if (!layer_range_ok(c, layer0, nlayers)) return THINK_ERR_INVALID_ARG;
   const Geometry& g = c->g;

@@ -48,9 +48,6 @@ struct ScoreParams {
   int ncolblk, nsplit, RP;  // RP = rows in flight per CTA iteration
   int criterion;
   uint32_t* error;          // device error word (may be null)
-  // k_colnorm_flat only: all items laid end to end, one unit per token row
-  const int64_t* row_cum;   // [B + 1] prompt rows of the batch entries before b
-  long long flat_rows;      // nlayers * ncolblk * row_cum[B]
 };
 
 struct CompactParams {
@@ -63,6 +60,8 @@ struct CompactParams {
   int B, L, N_kv, D, T, Tp, R;   // Tp = rows stored per thin tile (T padded to 8 for bf16)
   int re_cap;                    // tiles reserved per head after the prompt's thin tiles (re-pruned tail blocks)
   int layer0, nlayers;
+  int max_tiles;                 // longest pruned prefix of the batch, in tiles
+  int heads_first;               // CTA order of the bf16 kernel (set by the launcher)
 };
 
 struct RepruneParams {       // 64-token blocks of the unpruned tail -> thinned tiles (bf16)
@@ -160,8 +159,6 @@ struct DecodeParams {
 // launchers (one per translation unit); return the launch status
 cudaError_t launch_score(const ScoreParams& p, int dtype, cudaStream_t s);
 int score_ctas_per_sm(int dtype, int criterion);
-cudaError_t launch_score_flat(const ScoreParams& p, int dtype, int grid, cudaStream_t s);
-int score_flat_ctas_per_sm(int dtype, int criterion);
 cudaError_t launch_compact(const CompactParams& p, int dtype, int max_tiles, cudaStream_t s);
 cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t s, bool overlap_previous = false);
 cudaError_t launch_reprune(const RepruneParams& p, cudaStream_t s);

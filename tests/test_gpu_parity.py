@@ -386,6 +386,36 @@ def test_exact_ties_go_to_lower_channel():
     assert (sc[..., 3] == sc[..., 40]).all()
 
 
+def test_non_finite_keys_raise_the_error_word_and_stay_in_bounds():
+    """A NaN in one key column makes that channel's score NaN.  The ranking must still keep exactly T
+    channels per head (guard bytes behind every idx row survive) and the device error word must say so."""
+    from paper_2407_21018_b200 import binding as tk
+    w = wl.shrink(wl.get_config("c2"), S=500, L=2, steps=1)
+    data = wl.make_prefill(w, device="cpu")
+    K = data["K"].clone()
+    K[0, 17, 1, 3, 40] = float("nan")                      # layer 1, key head 3, channel 40
+    K[0, 18, 0, 5, 7] = float("inf")                       # layer 0, key head 5, channel 7
+    cache = make_cache(w, 1)
+    cache.idx.fill_(0xEE)
+    cache.score_select(data["Q_obs"].cuda(), K.cuda())
+    torch.cuda.synchronize()
+    assert cache.device_error() & tk.ERR_BIT_NON_FINITE
+    idx = cache.idx_tensor().cpu().numpy().astype(np.int64)
+    assert (np.diff(idx, axis=-1) > 0).all() and idx.max() < w.D          # T distinct channels in every head
+    n = w.B * w.L * w.N_kv * cache.T
+    assert (cache.idx[n:] == 0xEE).all()                                    # nothing written past the last row
+    assert 40 not in idx[0, 1, 3]                                           # the NaN channel ranks lowest
+    assert 7 in idx[0, 0, 5]                                                # an infinite score ranks highest
+    # untouched heads select what they select without the planted values
+    ref = make_cache(w, 1)
+    ref.score_select(data["Q_obs"].cuda(), data["K"].cuda())
+    torch.cuda.synchronize()
+    assert ref.device_error() == 0
+    keep = np.ones((w.L, w.N_kv), dtype=bool)
+    keep[1, 3] = keep[0, 5] = False
+    assert (idx[0][keep] == ref.idx_tensor().cpu().numpy().astype(np.int64)[0][keep]).all()
+
+
 def test_layer_ranges_and_determinism():
     """Per-layer calls give the same bytes as one call over all layers, and a repeat is identical."""
     w = wl.shrink(wl.get_config("c2"), S=900, L=3, steps=2)
@@ -467,6 +497,33 @@ def test_state_machine_and_capacity():
     assert e.value.status == tk.ERR_CAPACITY
     assert c.tail_len() == w.recent + 2
     torch.cuda.synchronize()
+    assert c.device_error() == 0
+
+
+def test_new_prompt_on_the_same_handle_reborrows_the_values():
+    """A second prefill with a different V view is a new prompt: it is accepted, the layers it does not cover
+    count as not compacted until they are, and decode then reads the NEW values."""
+    from paper_2407_21018_b200 import binding as tk
+    w = wl.shrink(wl.get_config("c2"), S=700, L=2, steps=2)
+    data = wl.make_prefill(w, device="cuda")
+    K, V, Q = data["K"], data["V"], data["Q_obs"]
+    st = wl.make_step(w, 0, device="cuda")
+    c = make_cache(w, 2)
+    c.prefill(Q, K, V)
+    V2 = (V.float() * 0.5).to(V.dtype)                      # same shape, other storage, other numbers
+    c.prefill(Q, K, V2, layer0=0, nlayers=1)                # covers layer 0 only
+    with pytest.raises(tk.ThinKError) as e:
+        c.append(st["k_new"], st["v_new"])                  # layer 1 still belongs to the old prompt
+    assert e.value.status == tk.ERR_STATE
+    c.prefill(Q, K, V2, layer0=1, nlayers=1)
+    c.append(st["k_new"], st["v_new"])
+    out = c.decode_attn(st["q"])
+    fresh = make_cache(w, 2)
+    fresh.prefill(Q, K, V2)
+    fresh.append(st["k_new"], st["v_new"])
+    want = fresh.decode_attn(st["q"])
+    torch.cuda.synchronize()
+    assert torch.equal(out, want)
     assert c.device_error() == 0
 
 
