@@ -108,6 +108,16 @@ def test_score_invariances():
     assert (orc.select_top_T(orc.score_closed_form(Q, 0.25 * K), T) == base).all()
 
 
+def test_cache_elements_with_decoded_tokens_hand_value():
+    # Sec. 3.3 by hand: one head, D = 4, half the channels kept, a prompt of 10 tokens of which the last 2 stay
+    # unpruned, 3 tokens decoded.  Keys: 8 pruned rows x 2 channels + (2 + 3) full rows x 4 = 16 + 20 = 36;
+    # values: (10 + 3) rows x 4 = 52; total 88.  Two layers of three heads: x 6 = 528.
+    assert orc.think_cache_elements([10], 1, 1, 4, keep=0.5, S_recent=2, new_tokens=3) == 88.0
+    assert orc.think_cache_elements([10], 2, 3, 4, keep=0.5, S_recent=2, new_tokens=3) == 528.0
+    # two sequences add up; without decoded tokens the tail holds the recent rows only
+    assert orc.think_cache_elements([10, 6], 1, 1, 4, keep=0.5, S_recent=2, new_tokens=0) == (16 + 8 + 40) + (8 + 8 + 24)
+
+
 def test_gqa_group_is_stacked_rows():
     # declared reading: the group's query heads are stacked; equals sqrt of summed squares
     rng = np.random.default_rng(9)
@@ -122,6 +132,14 @@ def test_magnitude_score_matches_library_norm():
     K = rng.normal(size=(31, 9))
     for p in (1, 2):
         np.testing.assert_allclose(orc.score_magnitude(K, p), np.linalg.norm(K, ord=p, axis=0), rtol=1e-13)
+
+
+def test_magnitude_score_hand_values():
+    # Eq. 1 on a 3 x 2 matrix worked by hand: column 0 = (3, -4, 0), column 1 = (1, 2, -2)
+    K = np.array([[3.0, 1.0], [-4.0, 2.0], [0.0, -2.0]])
+    assert orc.score_magnitude(K, 1).tolist() == [7.0, 5.0]        # |3| + |-4| + 0, 1 + 2 + 2
+    assert orc.score_magnitude(K, 2).tolist() == [5.0, 3.0]        # sqrt(9 + 16), sqrt(1 + 4 + 4)
+    # a transposed operand or a norm over the wrong axis gives (4, 6, 2) / (sqrt 10, sqrt 20, 2) instead
 
 
 # ------------------------------------------------------------------ top-T
