@@ -247,6 +247,58 @@ __global__ void __launch_bounds__(256) k_tail_write(const TailWriteParams p) {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// Seed of the unpruned tail at prefill (paper Sec. 3.3: the most recent prompt tokens keep every channel), bf16,
+// prompt order, values stored as they are.  One CTA moves up to 64 recent rows of one head: the key rows are staged
+// in shared memory and leave as whole 16-token steps of the fragment-order tail tile -- a lane builds one 16-byte
+// piece, a warp writes 512 contiguous bytes -- instead of one scattered 4-byte store per channel pair; the value
+// rows are copied 16 bytes per thread.  Rows of the last step beyond S_recent are written as zeros (the appends
+// that follow overwrite them one token at a time).
+__global__ void __launch_bounds__(128) k_tail_seed_bf16(const TailWriteParams p) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int D = p.D, pitch = D * 2 + 16, cpr = D / 8;
+  const int chunk = blockIdx.x, h = blockIdx.y;
+  const int b = blockIdx.z / p.nlayers, l = p.layer0 + blockIdx.z % p.nlayers;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
+  const int row0 = chunk * kTileTokens;                       // first tail position of this CTA
+  const int nrows = min(kTileTokens, p.R - row0);
+  const int64_t srow0 = (int64_t)p.seq_len[b] - p.R + row0;   // its source row
+  const __nv_bfloat16* ks = (const __nv_bfloat16*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn;
+  const __nv_bfloat16* vs = (const __nv_bfloat16*)p.v.ptr + b * p.v.sb + (int64_t)l * p.v.sl + (int64_t)h * p.v.sn;
+  const uint32_t s_addr = (uint32_t)__cvta_generic_to_shared(smem);
+  const int nsteps = (nrows + 15) >> 4;
+  for (int i = tid; i < nsteps * 16 * cpr; i += 128) {
+    const int r = i / cpr, ck = i % cpr;
+    const bool ok = r < nrows;
+    const void* g = ks + (srow0 + (ok ? r : 0)) * p.k.ss + ck * 8;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(s_addr + r * pitch + ck * 16), "l"(g), "r"(ok ? 16 : 0) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  for (int i = tid; i < nrows * cpr; i += 128) {
+    const int r = i / cpr, ck = i % cpr;
+    const uint4 v = __ldg((const uint4*)(vs + (srow0 + r) * p.v.ss + ck * 8));
+    *(uint4*)((__nv_bfloat16*)p.tail_v + (unit * p.cap + row0 + r) * D + ck * 8) = v;
+  }
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  __syncthreads();
+  unsigned char* tile = (unsigned char*)p.tail_k + (unit * p.tail_tiles_cap + chunk) * (int64_t)D * 128;
+  const int r8 = lane >> 2, q = lane & 3, ng = D >> 4;
+  for (int item = warp; item < nsteps * ng; item += 4) {
+    const int step = item / ng, s = item % ng;
+    const unsigned char* rowA = smem + (step * 16 + r8) * pitch + (16 * s + 2 * q) * 2;
+    const unsigned char* rowB = rowA + 8 * pitch;
+    uint4 v;
+    v.x = *(const uint32_t*)rowA;            // channels 16s + 2q, + 1 of token 16 * step + r8
+    v.y = *(const uint32_t*)(rowA + 16);     // channels 16s + 2q + 8, + 9
+    v.z = *(const uint32_t*)rowB;            // the same of token + 8
+    v.w = *(const uint32_t*)(rowB + 16);
+    *(uint4*)(tile + step * (D * 32) + s * 512 + lane * 16) = v;
+  }
+  // as in k_tail_write: launched beside the compaction kernel, this grid must not complete before the grid ahead of it
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Value-channel pruning (paper App. D): V_T[t][c] = V[t][perm_v[c]] for c < T_v, rows of Tvp elements
 // (zero padded), t < S_p.  A CTA stages 64 value rows of one head in shared memory (cp.async, padded
 // pitch); a thread then owns one 16-byte piece of the thinned rows -- its eight source channels stay in
@@ -390,6 +442,21 @@ cudaError_t launch_tail_write(const TailWriteParams& p, int dtype, cudaStream_t 
   if (total <= 0) return cudaSuccess;
   int blocks = (int)((total + 255) / 256);
   if (blocks > kSMs * 16) blocks = kSMs * 16;
+  if (dtype == THINK_BF16 && p.rows_from_seq_len && !p.tok.rows && !p.perm_v && p.pos0 == 0 && p.nrows == p.R &&
+      p.B * p.nlayers <= 65535 && p.N_kv <= 65535) {
+    // the prefill seed in prompt order: whole fragment-order steps per CTA
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((p.R + kTileTokens - 1) / kTileTokens, p.N_kv, p.B * p.nlayers);
+    cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = (size_t)kTileTokens * (p.D * 2 + 16);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap_previous ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, k_tail_seed_bf16, p);
+  }
   if (overlap_previous && dtype == THINK_BF16) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(blocks);
