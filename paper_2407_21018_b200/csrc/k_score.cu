@@ -81,27 +81,21 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
     }
   };
 
+  // The window rows of the G query heads that share key head h (stacked).  The first two rows of this thread
+  // are fetched now and summed after the key pass, so their latency runs under the key loads.
+  const bool with_q = active && p.criterion == THINK_SCORE_QUERY_DRIVEN;
+  const int q_rows = p.S_obs * p.G, q_step = p.nsplit * p.RP;
+  const Tin* qb = (const Tin*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl + j0;
+  auto q_row = [&](int rr) -> uint4 {
+    const int s = rr / p.G, g = rr % p.G;
+    return ldg16(qb + (int64_t)s * p.q.ss + (int64_t)(h * p.G + g) * p.q.sn);
+  };
+  uint4 q_early[2];
   {
-    // the window rows of the G query heads that share key head h (stacked)
-    double qacc[CH];
+    const int rr0 = split * p.RP + rl;
 #pragma unroll
-    for (int i = 0; i < CH; ++i) qacc[i] = 0.0;
-    if (active && p.criterion == THINK_SCORE_QUERY_DRIVEN) {
-      const Tin* qb = (const Tin*)p.q.ptr + b * p.q.sb + (int64_t)l * p.q.sl + j0;
-      const int nrows = p.S_obs * p.G;
-      for (int rr = split * p.RP + rl; rr < nrows; rr += p.nsplit * p.RP) {
-        int s = rr / p.G, g = rr % p.G;
-        uint4 v = ldg16(qb + (int64_t)s * p.q.ss + (int64_t)(h * p.G + g) * p.q.sn);
-        float x[CH];
-        Chunk<Tin>::unpack(v, x);
-#pragma unroll
-        for (int i = 0; i < CH; ++i) {
-          double d = (double)x[i];
-          qacc[i] = fma(d, d, qacc[i]);
-        }
-      }
-    }
-    reduce_store(qacc, 1);
+    for (int u = 0; u < 2; ++u)
+      q_early[u] = (with_q && rr0 + u * q_step < q_rows) ? q_row(rr0 + u * q_step) : make_uint4(0, 0, 0, 0);
   }
 
   double kacc[CH];
@@ -156,6 +150,26 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
       }
     }
   }
+  {
+    double qacc[CH];
+#pragma unroll
+    for (int i = 0; i < CH; ++i) qacc[i] = 0.0;
+    auto add_q = [&](const uint4& v) {
+      float x[CH];
+      Chunk<Tin>::unpack(v, x);
+#pragma unroll
+      for (int i = 0; i < CH; ++i) {
+        const double d = (double)x[i];
+        qacc[i] = fma(d, d, qacc[i]);
+      }
+    };
+    if (with_q) {
+      add_q(q_early[0]);                               // a row that was not fetched is all zeros
+      add_q(q_early[1]);
+      for (int rr = split * p.RP + rl + 2 * q_step; rr < q_rows; rr += q_step) add_q(q_row(rr));
+    }
+    reduce_store(qacc, 1);
+  }
   reduce_store(kacc, 0);
 
   // ticket: the last CTA of this (b, l, column block) finishes the job
@@ -170,25 +184,29 @@ __global__ void __launch_bounds__(kScoreThreads, 3) k_colnorm_score_select(const
   const double* base = p.partials + (int64_t)(z * p.ncolblk + colblk) * p.nsplit * 2 * CBE;
   const int ncols = min(CBE, (p.NC - colblk * p.CB) * CH);
   __syncthreads();
-  for (int c = tid; c < ncols; c += kScoreThreads) {
-    // partials are added in split order; loads are batched so their latencies overlap
-    double kn = 0.0, qn = 0.0;
+  // Partials are added in split order.  A thread takes two neighbouring columns (one 16-byte load per split and
+  // sum) and keeps 8 splits of both sums in flight, so the merge is a few round trips to L2, not one per split.
+  for (int c = 2 * tid; c < ncols; c += 2 * kScoreThreads) {
+    double kn0 = 0.0, kn1 = 0.0, qn0 = 0.0, qn1 = 0.0;
     for (int s0 = 0; s0 < p.nsplit; s0 += 8) {
-      double kv[8], qv[8];
+      double2 kv[8], qv[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const bool on = s0 + u < p.nsplit;
-        kv[u] = on ? __ldcg(base + (int64_t)(s0 + u) * 2 * CBE + c) : 0.0;
-        qv[u] = on ? __ldcg(base + (int64_t)(s0 + u) * 2 * CBE + CBE + c) : 0.0;
+        const double* row = base + (int64_t)(on ? s0 + u : 0) * 2 * CBE + c;
+        kv[u] = on ? __ldcg((const double2*)row) : make_double2(0.0, 0.0);
+        qv[u] = on ? __ldcg((const double2*)(row + CBE)) : make_double2(0.0, 0.0);
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { kn += kv[u]; qn += qv[u]; }
+      for (int u = 0; u < 8; ++u) { kn0 += kv[u].x; kn1 += kv[u].y; qn0 += qv[u].x; qn1 += qv[u].y; }
     }
-    double sc;
-    if (p.criterion == THINK_SCORE_QUERY_DRIVEN) sc = sqrt(qn * kn);
-    else if (p.criterion == THINK_SCORE_KEY_L2) sc = sqrt(kn);
-    else sc = kn;
-    red[c] = sc;
+    auto score_of = [&](double qn, double kn) -> double {
+      if (p.criterion == THINK_SCORE_QUERY_DRIVEN) return sqrt(qn * kn);
+      if (p.criterion == THINK_SCORE_KEY_L2) return sqrt(kn);
+      return kn;
+    };
+    red[c] = score_of(qn0, kn0);
+    red[c + 1] = score_of(qn1, kn1);
   }
   __syncthreads();
   const int heads = ncols / p.D;

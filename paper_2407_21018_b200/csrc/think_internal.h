@@ -219,25 +219,42 @@ __device__ __forceinline__ int64_t token_row(const TokenMap& m, int64_t unit, in
 // ascending; with `rest`, out[T..D) = the other channels ascending (out is then a permutation).
 // A NaN score ranks as -infinity, so the order is total and exactly T channels are kept whatever
 // the inputs; a NaN or infinite score raises kErrNonFinite in *error (when given).
+// A lane holds the scores of its channels (j = lane, lane + 32, ...; D <= 128) in registers and walks
+// all k once, eight broadcast loads at a time, counting for its channels together.
 __device__ __forceinline__ void select_head(const double* s, int D, int T, uint8_t* out, int lane, bool rest,
                                             uint32_t* error = nullptr) {
-  int base = 0, base_rest = T;
+  constexpr int MAXJ = 4;                       // channels per lane: D <= 32 * MAXJ
+  double sj[MAXJ];
+  int rank[MAXJ];
   bool bad = false;
-  for (int j0 = 0; j0 < D; j0 += 32) {
-    int j = j0 + lane;
-    bool keep = false;
-    if (j < D) {
-      double sj = s[j];
-      bad |= !(fabs(sj) <= 1.7976931348623157e308);
-      if (!(sj == sj)) sj = -INFINITY;
-      int rank = 0;
-      for (int k = 0; k < D; ++k) {
-        double sk = s[k];
-        if (!(sk == sk)) sk = -INFINITY;
-        rank += (sk > sj) || (sk == sj && k < j);
-      }
-      keep = rank < T;
+#pragma unroll
+  for (int i = 0; i < MAXJ; ++i) {
+    const int j = lane + 32 * i;
+    double v = j < D ? s[j] : 0.0;
+    bad |= j < D && !(fabs(v) <= 1.7976931348623157e308);
+    if (!(v == v)) v = -INFINITY;
+    sj[i] = v;
+    rank[i] = 0;
+  }
+  for (int k0 = 0; k0 < D; k0 += 8) {
+    double sk[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      sk[u] = s[k0 + u];                        // D is a multiple of 8
+      if (!(sk[u] == sk[u])) sk[u] = -INFINITY;
     }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+#pragma unroll
+      for (int i = 0; i < MAXJ; ++i) rank[i] += (sk[u] > sj[i]) || (sk[u] == sj[i] && k0 + u < lane + 32 * i);
+    }
+  }
+  int base = 0, base_rest = T;
+#pragma unroll
+  for (int i = 0; i < MAXJ; ++i) {
+    const int j = lane + 32 * i;
+    if (32 * i >= D) break;
+    const bool keep = j < D && rank[i] < T;
     const unsigned m = __ballot_sync(0xffffffffu, keep);
     const unsigned below = (1u << lane) - 1u;
     if (keep) out[base + __popc(m & below)] = (uint8_t)j;
