@@ -161,6 +161,8 @@ def measure_config(args, name, passes, warm, dev, world, barrier, do_e2e, sample
     from paper_2407_21018_b200 import replicas
 
     w = wl.get_config(name)
+    if args.layers:
+        w = wl.shrink(w, L=args.layers)            # fewer layers of the same shape (profiler captures): not a bench workload
     if args.lam is not None:
         w = dataclasses.replace(w, lam=args.lam, name=f"{w.name}-lam{args.lam}")
     nsteps = args.decode_steps if args.decode_steps is not None else w.steps
@@ -595,6 +597,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-budget", type=float, default=12.0)
+    ap.add_argument("--layers", type=int, default=0,
+                    help="run the config with this many layers instead of its own (small case for ncu captures; the "
+                         "workload label carries the changed layer count)")
     ap.add_argument("--profile", action="store_true",
                     help="for runs under ncu: take --warmup literally (fewer launches before the captured ones)")
     args = ap.parse_args()
