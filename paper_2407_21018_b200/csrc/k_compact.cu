@@ -82,7 +82,8 @@ __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
   const int D = p.D, T = p.T, Tp = p.Tp;
   const int pitch = D * 2 + 16;
   unsigned char* s_in = smem;                                   // [64][pitch]
-  uint8_t* s_idx = smem + kTileTokens * pitch;                  // [Tp], padding channels -> 255
+  uint16_t* s_off = (uint16_t*)(smem + kTileTokens * pitch);    // [Tp]: byte offset of kept channel c inside a staged row;
+                                                                // padding channels point at the 16 zero bytes behind the row
   // Which CTAs run side by side.  heads_first: the same 64 tokens of neighbouring heads and layers -- in the
   // paper's B x S x L x N x D layout those rows are one contiguous stretch (L*N*D elements per token), which
   // pays when that stretch is short (grouped-query shapes).  Otherwise: consecutive tiles of one head, whose
@@ -107,45 +108,67 @@ __global__ void __launch_bounds__(128) k_compact_bf16(const CompactParams p) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   const int64_t unit = ((int64_t)b * p.L + l) * p.N_kv + h;
-  for (int c = tid; c < Tp; c += 128) s_idx[c] = c < T ? p.idx[unit * T + c] : 255;
+  for (int c = tid; c < Tp; c += 128) s_off[c] = (uint16_t)(c < T ? 2 * p.idx[unit * T + c] : 2 * D);
   const __nv_bfloat16* src = (const __nv_bfloat16*)p.k.ptr + b * p.k.sb + (int64_t)l * p.k.sl + (int64_t)h * p.k.sn;
-  const int cpr = D / 8;                 // 16-byte chunks per row
+  // The tile's rows arrive by bulk copies: one instruction per 2 * D-byte row (threads 0..nvalid-1 issue one each),
+  // all completing on one mbarrier; rows past the prefix are zeroed with plain stores.
+  __shared__ __align__(8) uint64_t s_bar;
+  const uint32_t bar = (uint32_t)__cvta_generic_to_shared(&s_bar);
   const uint32_t s_in_addr = (uint32_t)__cvta_generic_to_shared(s_in);
-  for (int i = tid; i < kTileTokens * cpr; i += 128) {
-    const int r = i / cpr, ck = i % cpr;
-    const bool ok = r < nvalid;          // rows past the prefix become zeros
-    const int64_t row = TOK ? token_row(p.tok, unit, tok0 + (ok ? r : 0)) : (int64_t)(tok0 + (ok ? r : 0));
-    const void* g = src + row * p.k.ss + ck * 8;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(s_in_addr + r * pitch + ck * 16), "l"(g), "r"(ok ? 16 : 0) : "memory");
+  if (tid == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  asm volatile("cp.async.commit_group;" ::: "memory");
-  asm volatile("cp.async.wait_group 0;" ::: "memory");
+  if (tid < kTileTokens) *(uint4*)(s_in + tid * pitch + 2 * D) = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < (kTileTokens - nvalid) * (D / 8); i += 128)
+    *(uint4*)(s_in + (nvalid + i / (D / 8)) * pitch + (i % (D / 8)) * 16) = make_uint4(0, 0, 0, 0);
   __syncthreads();
+  if (tid == 0) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(nvalid * D * 2) : "memory");
+  if (tid < nvalid) {
+    const int64_t row = TOK ? token_row(p.tok, unit, tok0 + tid) : (int64_t)(tok0 + tid);
+    const void* g = src + row * p.k.ss;
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(s_in_addr + tid * pitch), "l"(g), "r"(D * 2), "r"(bar) : "memory");
+  }
+  {
+    // bounded wait (about a second at most): on expiry the error word is raised and the tile is left unwritten
+    uint32_t done = 0;
+    const long long t_start = clock64();
+    while (!done) {
+      asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                   : "=r"(done) : "r"(bar) : "memory");
+      if (!done && clock64() - t_start > 2000000000LL) break;
+    }
+    if (!done) {
+      if (tid == 0 && p.error) atomicOr(p.error, kErrWaitTimeout);
+      return;
+    }
+  }
 
   const int64_t gtile = p.thin_tile_base[b] + (int64_t)(l * p.N_kv + h) * (ntiles + p.re_cap) + tile;
   unsigned char* dst = (unsigned char*)p.k_thin + gtile * Tp * 128 + warp * (Tp * 32);   // step = warp
+  // a lane's four source channels of a group come as two 32-bit loads of byte offsets (pairs are neighbours in s_off)
   const int r = lane >> 2, q = lane & 3;
   const unsigned char* rowA = s_in + (warp * 16 + r) * pitch;
   const unsigned char* rowB = rowA + 8 * pitch;
-  auto elem = [&](const unsigned char* row, int ch) -> uint32_t {
-    return ch == 255 ? 0u : (uint32_t)*(const uint16_t*)(row + ch * 2);
+  auto pair = [](const unsigned char* row, uint32_t oo) -> uint32_t {      // elements at byte offsets oo & 0xffff, oo >> 16
+    return (uint32_t)*(const uint16_t*)(row + (oo & 0xffffu)) | ((uint32_t)*(const uint16_t*)(row + (oo >> 16)) << 16);
   };
   const int n16 = Tp >> 4;
   for (int s = 0; s < n16; ++s) {
-    const int c0 = s_idx[16 * s + 2 * q], c1 = s_idx[16 * s + 2 * q + 1];
-    const int c8 = s_idx[16 * s + 2 * q + 8], c9 = s_idx[16 * s + 2 * q + 9];
+    const uint32_t o01 = *(const uint32_t*)(s_off + 16 * s + 2 * q), o89 = *(const uint32_t*)(s_off + 16 * s + 2 * q + 8);
     uint4 v;
-    v.x = elem(rowA, c0) | (elem(rowA, c1) << 16);
-    v.y = elem(rowA, c8) | (elem(rowA, c9) << 16);
-    v.z = elem(rowB, c0) | (elem(rowB, c1) << 16);
-    v.w = elem(rowB, c8) | (elem(rowB, c9) << 16);
+    v.x = pair(rowA, o01);
+    v.y = pair(rowA, o89);
+    v.z = pair(rowB, o01);
+    v.w = pair(rowB, o89);
     *(uint4*)(dst + s * 512 + lane * 16) = v;
   }
   if (Tp & 8) {
-    const int c0 = s_idx[16 * n16 + 2 * q], c1 = s_idx[16 * n16 + 2 * q + 1];
+    const uint32_t o01 = *(const uint32_t*)(s_off + 16 * n16 + 2 * q);
     uint2 v;
-    v.x = elem(rowA, c0) | (elem(rowA, c1) << 16);
-    v.y = elem(rowB, c0) | (elem(rowB, c1) << 16);
+    v.x = pair(rowA, o01);
+    v.y = pair(rowB, o01);
     *(uint2*)(dst + n16 * 512 + lane * 8) = v;
   }
 }
@@ -402,7 +425,7 @@ cudaError_t launch_compact(const CompactParams& p_in, int dtype, int max_tiles, 
   size_t smem = (size_t)kTileTokens * (p.D * E + 16) + (size_t)p.Tp * kTileTokens * E + ((p.T + 15) & ~15);
   cudaError_t e;
   if (dtype == THINK_BF16) {
-    smem = (size_t)kTileTokens * (p.D * 2 + 16) + ((p.Tp + 15) & ~15);
+    smem = (size_t)kTileTokens * (p.D * 2 + 16) + 2 * (size_t)((p.Tp + 15) & ~15);
     cudaLaunchConfig_t cfg = {};
     if (p.B > 65535 || p.nlayers > 65535) return cudaErrorInvalidValue;
     p.heads_first = p.N_kv * p.nlayers <= 256 && max_tiles <= 65535;

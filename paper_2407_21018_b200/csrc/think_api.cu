@@ -380,6 +380,7 @@ thinK_status compact_impl(thinK_cache* c, thinK_tensor5 k, thinK_tensor5 v, cons
   p.B = g.B; p.L = g.L; p.N_kv = g.N_kv; p.D = g.D; p.T = g.T; p.Tp = g.Tp; p.R = g.R;
   p.re_cap = g.tail_tiles_cap;
   p.layer0 = layer0; p.nlayers = nlayers;
+  p.error = (uint32_t*)(c->ws + c->w.error);
   if (launch_compact(p, g.dtype, g.max_thin_tiles, (cudaStream_t)stream) != cudaSuccess) return THINK_ERR_CUDA;
   if (g.vt) {
     CompactValueParams cv;

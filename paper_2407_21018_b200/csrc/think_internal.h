@@ -62,6 +62,7 @@ struct CompactParams {
   int layer0, nlayers;
   int max_tiles;                 // longest pruned prefix of the batch, in tiles
   int heads_first;               // CTA order of the bf16 kernel (set by the launcher)
+  uint32_t* error;               // device error word (may be null)
 };
 
 struct RepruneParams {       // 64-token blocks of the unpruned tail -> thinned tiles (bf16)
