@@ -313,8 +313,9 @@ int32_t thinK_repruned_len(const thinK_cache* c, int32_t layer);
 int32_t thinK_tail_len(const thinK_cache* c, int32_t layer);
 
 /* Reads the device-side error word (0 = none) with a synchronous copy.  Bits: 1 a kept-token index of
- * thinK_prefill_evicted was out of range; 2 a bounded wait inside a kernel ran out; 4 a kernel found its
- * shared memory misaligned; 8 a channel score was NaN or infinite (non-finite K or Q: exactly T channels
+ * thinK_prefill_evicted was out of range; 2 a bounded wait inside a kernel ran out (value-score kernel: that unit's
+ * selection is missing; compaction: a tile whose row copies did not complete within about a second is left
+ * unwritten -- re-create the cache); 4 a kernel found its shared memory misaligned; 8 a channel score was NaN or infinite (non-finite K or Q: exactly T channels
  * are still selected, NaN scores ranking lowest). */
 thinK_status thinK_device_error(thinK_cache* c, int32_t* out_code);
 
