@@ -301,7 +301,7 @@ def measure_config(args, name, passes, warm, dev, world, barrier, do_e2e, sample
             hK, hV, hQ = pin(K), pin(V), pin(Q)
             hs = [{k: pin(v) for k, v in s.items()} for s in steps_in]
             hout = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
-            n_e2e = max(1, min(passes, 3))
+            n_e2e = max(1, min(passes, 5))
             # Two sets of input tensors on the device: while pass i computes from one, the copy stream brings pass
             # i + 1's prompt and its per-step inputs into the other (what a server does with the next batch).  Every
             # pass still copies all its inputs -- the prompt tensors and every decode step's q, k_new, v_new -- from
